@@ -1,0 +1,233 @@
+"""CPU oracle for PPD -- test infrastructure only.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
+It shares no code with the CUDA library and never calls it.
+
+`Oracle` wraps the C implementation (oracle/ppd_oracle.c, double precision);
+`oracle.theory` holds the paper's latency/compute model (Section 4, Theorem 4.1).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libppd_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    src = os.path.join(_HERE, "ppd_oracle.c")
+    if force or not os.path.exists(_LIB_PATH) or os.path.getmtime(_LIB_PATH) < os.path.getmtime(src):
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", _LIB_PATH, src, "-lm"])
+    return _LIB_PATH
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab", "max_seq", "max_k")] + \
+               [("rms_eps", ctypes.c_double), ("rope_theta", ctypes.c_double), ("kv_round_bf16", ctypes.c_int32)]
+
+
+_P = ctypes.c_void_p
+_I = ctypes.c_int32
+_D = ctypes.c_double
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    lib = ctypes.CDLL(_LIB_PATH)
+    sig = {
+        "orc_create": (_P, [ctypes.POINTER(_Config), _P]),
+        "orc_destroy": (None, [_P]),
+        "orc_reset": (None, [_P]),
+        "orc_pos": (_I, [_P]),
+        "orc_times": (None, [_P, _P, _P]),
+        "orc_prefill": (ctypes.c_int, [_P, _P, _I]),
+        "orc_greedy_probe": (ctypes.c_int, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
+        "orc_ppd": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
+        "orc_embed": (None, [_P, _I, _P]),
+        "orc_layer": (None, [_P, _I, _P, _I, _I]),
+        "orc_head": (None, [_P, _P, _P]),
+        "orc_rmsnorm": (None, [_P, _P, _I, _D, _P]),
+        "orc_matvec": (None, [_P, _I, _I, _P, _P]),
+        "orc_rope": (None, [_P, _I, _I, _I, _D]),
+        "orc_silu": (_D, [_D]),
+        "orc_attention": (None, [_P, _P, _P, _I, _P, _P, _I, _I, _P]),
+        "orc_topk": (None, [_P, _I, _I, _P]),
+        "orc_round_bf16": (_D, [_D]),
+        "orc_bf16_to_double": (_D, [ctypes.c_uint16]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+# ----------------------------------------------------------------- primitive ops
+
+def rmsnorm(h, g_bf16, eps):
+    lib = _load()
+    h = _f64(h)
+    g = np.ascontiguousarray(g_bf16, dtype=np.uint16)
+    out = np.empty_like(h)
+    lib.orc_rmsnorm(_ptr(h), _ptr(g), h.size, eps, _ptr(out))
+    return out
+
+
+def matvec(w_bf16, x):
+    """y = W x with W a uint16 (bf16) array [N][K]."""
+    lib = _load()
+    w = np.ascontiguousarray(w_bf16, dtype=np.uint16)
+    x = _f64(x)
+    n, k = w.shape
+    assert x.shape == (k,)
+    y = np.empty(n, dtype=np.float64)
+    lib.orc_matvec(_ptr(w), n, k, _ptr(x), _ptr(y))
+    return y
+
+
+def rope(v, n_heads, head_dim, pos, theta):
+    lib = _load()
+    out = _f64(v).copy()
+    assert out.size == n_heads * head_dim
+    lib.orc_rope(_ptr(out), n_heads, head_dim, pos, theta)
+    return out
+
+
+def silu(z):
+    return _load().orc_silu(float(z))
+
+
+def attention(q, kc, vc, k_tail=None, v_tail=None, *, n_heads, head_dim):
+    """q [D]; kc, vc [T][D] canonical rows; optional one extra position k_tail/v_tail [D]."""
+    lib = _load()
+    q, kc, vc = _f64(q), _f64(kc), _f64(vc)
+    d = n_heads * head_dim
+    t = kc.shape[0] if kc.size else 0
+    kt = _f64(k_tail) if k_tail is not None else None
+    vt = _f64(v_tail) if v_tail is not None else None
+    out = np.empty(d, dtype=np.float64)
+    lib.orc_attention(_ptr(q), _ptr(kc), _ptr(vc), t, _ptr(kt), _ptr(vt), n_heads, head_dim, _ptr(out))
+    return out
+
+
+def topk(logits, k):
+    lib = _load()
+    lg = _f64(logits)
+    ids = np.empty(k, dtype=np.int32)
+    lib.orc_topk(_ptr(lg), lg.size, k, _ptr(ids))
+    return ids
+
+
+def round_bf16(x):
+    lib = _load()
+    return np.array([lib.orc_round_bf16(float(v)) for v in np.ravel(x)]).reshape(np.shape(x))
+
+
+# ----------------------------------------------------------------- model
+
+class Oracle:
+    """Double-precision reference decoder holding a bf16 weight blob (uint16 numpy array)."""
+
+    def __init__(self, shape, blob, max_seq, max_k=8, kv_round_bf16=True):
+        lib = _load()
+        self.shape = shape
+        self.blob = np.ascontiguousarray(blob, dtype=np.uint16)  # kept alive: the C side borrows it
+        assert self.blob.size == shape.blob_elems
+        self.cfg = _Config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn,
+                           shape.vocab, max_seq, max_k, shape.rms_eps, shape.rope_theta,
+                           1 if kv_round_bf16 else 0)
+        self._m = lib.orc_create(ctypes.byref(self.cfg), _ptr(self.blob))
+        if not self._m:
+            raise ValueError("orc_create failed (bad shape or out of memory)")
+        self._lib = lib
+
+    def close(self):
+        if getattr(self, "_m", None):
+            self._lib.orc_destroy(self._m)
+            self._m = None
+
+    __del__ = close
+
+    @property
+    def pos(self):
+        return self._lib.orc_pos(self._m)
+
+    def times(self):
+        a, b = ctypes.c_double(), ctypes.c_double()
+        self._lib.orc_times(self._m, ctypes.byref(a), ctypes.byref(b))
+        return a.value, b.value
+
+    def prefill(self, prompt):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        self._lib.orc_reset(self._m)
+        rc = self._lib.orc_prefill(self._m, _ptr(p), p.size)
+        if rc != 0:
+            raise ValueError(f"orc_prefill rc={rc}")
+
+    def greedy_probe(self, n, k=0, l=1, forced=None, dump_logits=False):
+        """Greedy decode n tokens; returns dict(tokens, hit, margin_final, margin_early[, final_logits,
+        early_logits, cand])."""
+        V = self.shape.vocab
+        tokens = np.empty(n, dtype=np.int32)
+        hit = np.zeros(n, dtype=np.uint8)
+        mf = np.empty(n, dtype=np.float64)
+        me = np.full(n, np.inf, dtype=np.float64)
+        fl = np.empty((n, V), dtype=np.float64) if dump_logits else None
+        el = np.empty((n, V), dtype=np.float64) if (dump_logits and k > 0) else None
+        cand = np.empty((n, k), dtype=np.int32) if k > 0 else None
+        f = np.ascontiguousarray(forced, dtype=np.int32) if forced is not None else None
+        if f is not None:
+            assert f.size >= n
+        rc = self._lib.orc_greedy_probe(self._m, n, k, l, _ptr(f), _ptr(tokens), _ptr(hit), _ptr(mf),
+                                        _ptr(me), _ptr(fl), _ptr(el), _ptr(cand))
+        if rc != 0:
+            raise ValueError(f"orc_greedy_probe rc={rc}")
+        return dict(tokens=tokens, hit=hit, margin_final=mf, margin_early=me, final_logits=fl,
+                    early_logits=el, cand=cand)
+
+    def ppd(self, n, k, l, eos=-1):
+        tokens = np.empty(n, dtype=np.int32)
+        hit = np.zeros(n, dtype=np.uint8)
+        n_out = ctypes.c_int32()
+        units, cunits = ctypes.c_int64(), ctypes.c_int64()
+        rc = self._lib.orc_ppd(self._m, n, k, l, eos, _ptr(tokens), _ptr(hit), ctypes.byref(n_out),
+                               ctypes.byref(units), ctypes.byref(cunits))
+        if rc != 0:
+            raise ValueError(f"orc_ppd rc={rc}")
+        m = n_out.value
+        return dict(tokens=tokens[:m], hit=hit[:m], units=units.value, cunits=cunits.value)
+
+    # building blocks (used by op-level parity tests)
+    def embed(self, token):
+        h = np.empty(self.shape.d_model, dtype=np.float64)
+        self._lib.orc_embed(self._m, int(token), _ptr(h))
+        return h
+
+    def layer(self, layer, h, pos, slot=-1):
+        h = _f64(h).copy()
+        self._lib.orc_layer(self._m, layer, _ptr(h), pos, slot)
+        return h
+
+    def head(self, h):
+        h = _f64(h)
+        out = np.empty(self.shape.vocab, dtype=np.float64)
+        self._lib.orc_head(self._m, _ptr(h), _ptr(out))
+        return out

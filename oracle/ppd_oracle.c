@@ -1,0 +1,459 @@
+/*
+ * CPU oracle for Predictive Pipelined Decoding (PPD) -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, obviously-correct implementation of what the GPU decode path computes:
+ * a LLaMA-shaped decoder (RMSNorm, rotate-half RoPE, multi-head causal attention with a
+ * KV cache, SwiGLU FFN, untied unembedding), greedy decoding with an early-layer probe,
+ * and the PPD state machine of the paper's Algorithm 2 (Algorithm 1 is the case where the
+ * early layer is d/2).  It shares no code with the CUDA library; only tests, the smoke
+ * check and the benchmark's CPU-baseline leg may load it.
+ *
+ * Arithmetic: weights are bf16 values (given as a uint16 blob) widened exactly; all
+ * activations, sums and transcendental functions are IEEE double.  K and V are rounded to
+ * bf16 (round-to-nearest-even) when stored into the cache, because the cache's storage
+ * format is part of the model definition; this can be switched off (kv_round_bf16 = 0).
+ * There is no blocking, fusion or reordering: each function is the textbook definition.
+ * OpenMP only distributes independent output rows / heads over threads.
+ *
+ * Notation (paper -> here): d = n_layers; the early-prediction layer (paper: d-bar) is
+ * `l`; the number of generated tokens (paper: l) is `n`; k = number of early candidates;
+ * b = min(l, d-l) = layers a candidate branch runs before it is verified (the paper
+ * assumes l >= d/2, where b = d-l).
+ *
+ * Pins (see tests): logits against an independent float64 PyTorch composition and the
+ * Hugging Face LLaMA module on the same blob; PPD tokens == greedy tokens and PPD hit flags
+ * == probe flags for every (k, l) (the paper's exactness claim, Section 3); latency /
+ * compute units against Theorem 4.1 with the realised hit count; top-k against a sort.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <time.h>
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab, max_seq, max_k;
+    double rms_eps, rope_theta;
+    int32_t kv_round_bf16;
+} orc_config;
+
+typedef struct {
+    const uint16_t *g1, *wq, *wk, *wv, *wo, *g2, *wg, *wu, *wd;
+} orc_layer_w;
+
+typedef struct orc_model {
+    orc_config c;
+    const uint16_t* emb;
+    const uint16_t* g_final;
+    const uint16_t* w_head;
+    orc_layer_w* lw;
+    double *kc, *vc;  /* canonical cache  [layer][max_seq][D] */
+    double *kb, *vb;  /* branch slots     [max_k][layer][D]   */
+    int32_t pos;      /* position of the pending token = number of cached positions */
+    int32_t pending;  /* token to be fed at `pos`; -1 before prefill */
+    double t_layers, t_heads; /* wall seconds spent in layers / heads (reporting only) */
+} orc_model;
+
+static double now_s(void) {
+    struct timespec ts;
+    clock_gettime(CLOCK_MONOTONIC, &ts);
+    return (double)ts.tv_sec + 1e-9 * (double)ts.tv_nsec;
+}
+
+/* ------------------------------------------------------------------ primitives */
+
+double orc_bf16_to_double(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+/* Round a double to the nearest bf16 value (ties to even), returned as double. */
+double orc_round_bf16(double x) {
+    if (x == 0.0 || !isfinite(x)) return x;
+    int e;
+    double m = frexp(x, &e);            /* x = m * 2^e, 0.5 <= |m| < 1 */
+    if (e < -125) {                     /* below the normal range: fixed quantum 2^-133 */
+        double q = ldexp(1.0, -133);
+        return nearbyint(x / q) * q;
+    }
+    double scaled = ldexp(m, 8);        /* 8 significant bits: 128 <= |scaled| < 256 */
+    return ldexp(nearbyint(scaled), e - 8); /* default rounding mode = ties to even */
+}
+
+/* out_i = g_i * h_i / sqrt(mean(h^2) + eps) */
+void orc_rmsnorm(const double* h, const uint16_t* g, int D, double eps, double* out) {
+    double ss = 0.0;
+    for (int i = 0; i < D; ++i) ss += h[i] * h[i];
+    double inv = 1.0 / sqrt(ss / (double)D + eps);
+    for (int i = 0; i < D; ++i) out[i] = orc_bf16_to_double(g[i]) * (h[i] * inv);
+}
+
+/* y[n] = sum_k W[n][k] x[k],  W row-major [N][K] in bf16 */
+void orc_matvec(const uint16_t* W, int N, int K, const double* x, double* y) {
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        const uint16_t* w = W + (size_t)n * (size_t)K;
+        double acc = 0.0;
+        for (int k = 0; k < K; ++k) acc += orc_bf16_to_double(w[k]) * x[k];
+        y[n] = acc;
+    }
+}
+
+/* Rotate-half RoPE on v[H][hd]: dims i and i+hd/2 form a pair rotated by pos * theta^(-2i/hd). */
+void orc_rope(double* v, int H, int hd, int pos, double theta) {
+    int half = hd / 2;
+    for (int h = 0; h < H; ++h) {
+        double* p = v + (size_t)h * hd;
+        for (int i = 0; i < half; ++i) {
+            double ang = (double)pos * pow(theta, -2.0 * (double)i / (double)hd);
+            double c = cos(ang), s = sin(ang);
+            double a = p[i], b = p[i + half];
+            p[i] = a * c - b * s;
+            p[i + half] = b * c + a * s;
+        }
+    }
+}
+
+double orc_silu(double z) { return z / (1.0 + exp(-z)); }
+
+/*
+ * Causal attention for one query token.  Keys/values: n_canon rows of kc/vc (row stride D),
+ * followed, when k_tail != NULL, by one more position held in k_tail/v_tail ([D] each).
+ * out[h*hd + j] = sum_t softmax_t(q_h . K_t,h / sqrt(hd)) V_t,h,j
+ */
+void orc_attention(const double* q, const double* kc, const double* vc, int n_canon,
+                   const double* k_tail, const double* v_tail, int H, int hd, double* out) {
+    const int D = H * hd;
+    const int T = n_canon + (k_tail ? 1 : 0);
+    const double scale = 1.0 / sqrt((double)hd);
+#pragma omp parallel for schedule(static)
+    for (int h = 0; h < H; ++h) {
+        double* s = (double*)malloc(sizeof(double) * (size_t)T);
+        const double* qh = q + (size_t)h * hd;
+        double mx = -INFINITY;
+        for (int t = 0; t < T; ++t) {
+            const double* kt = (t < n_canon ? kc + (size_t)t * D : k_tail) + (size_t)h * hd;
+            double acc = 0.0;
+            for (int j = 0; j < hd; ++j) acc += qh[j] * kt[j];
+            s[t] = acc * scale;
+            if (s[t] > mx) mx = s[t];
+        }
+        double den = 0.0;
+        for (int t = 0; t < T; ++t) { s[t] = exp(s[t] - mx); den += s[t]; }
+        for (int j = 0; j < hd; ++j) {
+            double acc = 0.0;
+            for (int t = 0; t < T; ++t) {
+                const double* vt = (t < n_canon ? vc + (size_t)t * D : v_tail) + (size_t)h * hd;
+                acc += (s[t] / den) * vt[j];
+            }
+            out[(size_t)h * hd + j] = acc;
+        }
+        free(s);
+    }
+}
+
+/* ids[0..k) = the k largest logits, ordered by (value descending, id ascending). */
+void orc_topk(const double* logits, int V, int k, int32_t* ids) {
+    for (int r = 0; r < k; ++r) {
+        int best = -1;
+        for (int v = 0; v < V; ++v) {
+            int taken = 0;
+            for (int j = 0; j < r; ++j) if (ids[j] == v) { taken = 1; break; }
+            if (taken) continue;
+            if (best < 0 || logits[v] > logits[best]) best = v; /* strict > keeps the lowest id on ties */
+        }
+        ids[r] = best;
+    }
+}
+
+/* ------------------------------------------------------------------ model */
+
+size_t orc_blob_elems(const orc_config* c) {
+    size_t D = (size_t)c->d_model, F = (size_t)c->d_ffn, V = (size_t)c->vocab;
+    return V * D + (size_t)c->n_layers * (2 * D + 4 * D * D + 3 * F * D) + D + V * D;
+}
+
+/* The blob is borrowed: the caller keeps it alive for the model's lifetime. */
+orc_model* orc_create(const orc_config* c, const uint16_t* blob) {
+    if (!c || !blob || c->n_layers < 1 || c->n_heads * c->head_dim != c->d_model ||
+        (c->head_dim & 1) || c->max_seq < 2 || c->max_k < 0)
+        return NULL;
+    orc_model* m = (orc_model*)calloc(1, sizeof(orc_model));
+    m->c = *c;
+    size_t D = (size_t)c->d_model, F = (size_t)c->d_ffn, V = (size_t)c->vocab;
+    const uint16_t* p = blob;
+    m->emb = p; p += V * D;
+    m->lw = (orc_layer_w*)calloc((size_t)c->n_layers, sizeof(orc_layer_w));
+    for (int l = 0; l < c->n_layers; ++l) {
+        orc_layer_w* w = &m->lw[l];
+        w->g1 = p; p += D;
+        w->wq = p; p += D * D;
+        w->wk = p; p += D * D;
+        w->wv = p; p += D * D;
+        w->wo = p; p += D * D;
+        w->g2 = p; p += D;
+        w->wg = p; p += F * D;
+        w->wu = p; p += F * D;
+        w->wd = p; p += D * F;
+    }
+    m->g_final = p; p += D;
+    m->w_head = p;
+    size_t cache = (size_t)c->n_layers * (size_t)c->max_seq * D;
+    size_t slots = (size_t)(c->max_k > 0 ? c->max_k : 1) * (size_t)c->n_layers * D;
+    m->kc = (double*)calloc(cache, sizeof(double));
+    m->vc = (double*)calloc(cache, sizeof(double));
+    m->kb = (double*)calloc(slots, sizeof(double));
+    m->vb = (double*)calloc(slots, sizeof(double));
+    m->pos = 0;
+    m->pending = -1;
+    if (!m->kc || !m->vc || !m->kb || !m->vb) return NULL;
+    return m;
+}
+
+void orc_destroy(orc_model* m) {
+    if (!m) return;
+    free(m->kc); free(m->vc); free(m->kb); free(m->vb); free(m->lw); free(m);
+}
+
+void orc_reset(orc_model* m) { m->pos = 0; m->pending = -1; m->t_layers = m->t_heads = 0.0; }
+int32_t orc_pos(const orc_model* m) { return m->pos; }
+void orc_times(const orc_model* m, double* t_layers, double* t_heads) {
+    *t_layers = m->t_layers; *t_heads = m->t_heads;
+}
+
+void orc_embed(const orc_model* m, int32_t token, double* h) {
+    int D = m->c.d_model;
+    const uint16_t* e = m->emb + (size_t)token * D;
+    for (int i = 0; i < D; ++i) h[i] = orc_bf16_to_double(e[i]);
+}
+
+/*
+ * One decoder block applied in place to the residual stream h of a token at position `pos`.
+ * slot < 0 : the token is on the committed path; its K/V go to the canonical cache at `pos`
+ *            and it attends to canonical positions 0..pos.
+ * slot >= 0: the token is candidate `slot` of a speculative branch; its K/V go to that
+ *            branch slot and it attends to canonical positions 0..pos-1 plus its own slot.
+ */
+void orc_layer(orc_model* m, int layer, double* h, int pos, int slot) {
+    const orc_config* c = &m->c;
+    const int D = c->d_model, F = c->d_ffn, H = c->n_heads, hd = c->head_dim;
+    const orc_layer_w* w = &m->lw[layer];
+    double t0 = now_s();
+    double* n = (double*)malloc(sizeof(double) * D);
+    double* q = (double*)malloc(sizeof(double) * D);
+    double* k = (double*)malloc(sizeof(double) * D);
+    double* v = (double*)malloc(sizeof(double) * D);
+    double* a = (double*)malloc(sizeof(double) * D);
+    double* o = (double*)malloc(sizeof(double) * D);
+    double* gt = (double*)malloc(sizeof(double) * F);
+    double* up = (double*)malloc(sizeof(double) * F);
+
+    orc_rmsnorm(h, w->g1, D, c->rms_eps, n);
+    orc_matvec(w->wq, D, D, n, q);
+    orc_matvec(w->wk, D, D, n, k);
+    orc_matvec(w->wv, D, D, n, v);
+    orc_rope(q, H, hd, pos, c->rope_theta);
+    orc_rope(k, H, hd, pos, c->rope_theta);
+    if (c->kv_round_bf16)
+        for (int i = 0; i < D; ++i) { k[i] = orc_round_bf16(k[i]); v[i] = orc_round_bf16(v[i]); }
+
+    double* kc = m->kc + (size_t)layer * c->max_seq * D;
+    double* vc = m->vc + (size_t)layer * c->max_seq * D;
+    if (slot < 0) {
+        memcpy(kc + (size_t)pos * D, k, sizeof(double) * D);
+        memcpy(vc + (size_t)pos * D, v, sizeof(double) * D);
+        orc_attention(q, kc, vc, pos + 1, NULL, NULL, H, hd, a);
+    } else {
+        double* kb = m->kb + ((size_t)slot * c->n_layers + layer) * D;
+        double* vb = m->vb + ((size_t)slot * c->n_layers + layer) * D;
+        memcpy(kb, k, sizeof(double) * D);
+        memcpy(vb, v, sizeof(double) * D);
+        orc_attention(q, kc, vc, pos, kb, vb, H, hd, a);
+    }
+    orc_matvec(w->wo, D, D, a, o);
+    for (int i = 0; i < D; ++i) h[i] += o[i];
+
+    orc_rmsnorm(h, w->g2, D, c->rms_eps, n);
+    orc_matvec(w->wg, F, D, n, gt);
+    orc_matvec(w->wu, F, D, n, up);
+    for (int i = 0; i < F; ++i) gt[i] = orc_silu(gt[i]) * up[i];
+    orc_matvec(w->wd, D, F, gt, o);
+    for (int i = 0; i < D; ++i) h[i] += o[i];
+
+    free(n); free(q); free(k); free(v); free(a); free(o); free(gt); free(up);
+    m->t_layers += now_s() - t0;
+}
+
+/* logits = W_H . RMSNorm_final(h).  Used for the final head and, unchanged, for the early
+ * head (the untrained-classifier variant of the paper's Table 2, column "N"). */
+void orc_head(orc_model* m, const double* h, double* logits) {
+    double t0 = now_s();
+    int D = m->c.d_model;
+    double* n = (double*)malloc(sizeof(double) * D);
+    orc_rmsnorm(h, m->g_final, D, m->c.rms_eps, n);
+    orc_matvec(m->w_head, m->c.vocab, D, n, logits);
+    free(n);
+    m->t_heads += now_s() - t0;
+}
+
+/* gap between the r-th and (r+1)-th largest logits (r counted from 1) */
+static double margin_at(const double* logits, int V, int r) {
+    if (r + 1 > V) return INFINITY;
+    int32_t* ids = (int32_t*)malloc(sizeof(int32_t) * (size_t)(r + 1));
+    orc_topk(logits, V, r + 1, ids);
+    double g = logits[ids[r - 1]] - logits[ids[r]];
+    free(ids);
+    return g;
+}
+
+/*
+ * Prompt convention: the last prompt token is the start token x_0 of the decode loop.
+ * Positions 0..P-2 are run through all layers to fill the cache; prompt[P-1] stays pending
+ * and is fed by the first decode step at position P-1.
+ */
+int orc_prefill(orc_model* m, const int32_t* prompt, int32_t P) {
+    if (P < 1 || P > m->c.max_seq) return -1;
+    for (int i = 0; i < P; ++i) if (prompt[i] < 0 || prompt[i] >= m->c.vocab) return -1;
+    double* h = (double*)malloc(sizeof(double) * m->c.d_model);
+    m->pos = 0;
+    for (int t = 0; t + 1 < P; ++t) {
+        orc_embed(m, prompt[t], h);
+        for (int l = 0; l < m->c.n_layers; ++l) orc_layer(m, l, h, t, -1);
+    }
+    free(h);
+    m->pos = P - 1;
+    m->pending = prompt[P - 1];
+    return 0;
+}
+
+/*
+ * Conventional greedy decoding (all d layers, argmax of the final logits) with a probe of
+ * the early head after layer l: hit[s] = 1 iff the final argmax of step s is among the
+ * top-k tokens of the early logits -- the paper's definition of a match.
+ *
+ * forced (optional, [n]): token fed at step s+1 instead of the model's own argmax (teacher
+ * forcing for parity runs); tokens[] always reports the model's own argmax.
+ * Optional dumps (may be NULL): final_logits/early_logits [n][V], cand [n][k],
+ * margin_final [n] (top-1 minus top-2), margin_early [n] (k-th minus (k+1)-th early logit).
+ */
+int orc_greedy_probe(orc_model* m, int32_t n, int32_t k, int32_t l, const int32_t* forced,
+                     int32_t* tokens, uint8_t* hit, double* margin_final, double* margin_early,
+                     double* final_logits, double* early_logits, int32_t* cand) {
+    const orc_config* c = &m->c;
+    const int D = c->d_model, V = c->vocab, d = c->n_layers;
+    if (m->pending < 0 || n < 0 || k < 0 || k > V || l < 1 || l > d) return -1;
+    if (m->pos + n > c->max_seq) return -2;
+    double* h = (double*)malloc(sizeof(double) * D);
+    double* lf = (double*)malloc(sizeof(double) * V);
+    double* le = (double*)malloc(sizeof(double) * V);
+    int32_t* ids = (int32_t*)malloc(sizeof(int32_t) * (size_t)(k > 0 ? k : 1));
+    for (int s = 0; s < n; ++s) {
+        orc_embed(m, m->pending, h);
+        for (int j = 0; j < d; ++j) {
+            orc_layer(m, j, h, m->pos, -1);
+            if (j + 1 == l && k > 0) orc_head(m, h, le);
+        }
+        orc_head(m, h, lf);
+        int32_t next;
+        orc_topk(lf, V, 1, &next);
+        tokens[s] = next;
+        if (k > 0) {
+            orc_topk(le, V, k, ids);
+            uint8_t f = 0;
+            for (int i = 0; i < k; ++i) if (ids[i] == next) f = 1;
+            if (hit) hit[s] = f;
+            if (cand) memcpy(cand + (size_t)s * k, ids, sizeof(int32_t) * (size_t)k);
+            if (margin_early) margin_early[s] = margin_at(le, V, k);
+            if (early_logits) memcpy(early_logits + (size_t)s * V, le, sizeof(double) * V);
+        } else if (hit) hit[s] = 0;
+        if (margin_final) margin_final[s] = margin_at(lf, V, 1);
+        if (final_logits) memcpy(final_logits + (size_t)s * V, lf, sizeof(double) * V);
+        m->pending = forced ? forced[s] : next;
+        m->pos += 1;
+    }
+    free(h); free(lf); free(le); free(ids);
+    return 0;
+}
+
+/*
+ * The PPD state machine (Algorithm 2; Algorithm 1 when l = d/2).
+ *
+ * Per step: the main pass brings the current token to layer l (from layer 1 after a miss,
+ * from the committed hidden state at layer b after a hit), the early head proposes k
+ * candidates, each candidate runs layers 1..b at the next position against the shared
+ * prefix (in parallel with the main pass in the paper; here one after another), the main
+ * pass finishes layers l+1..d and takes the argmax, and the matching branch -- its hidden
+ * state and its K/V for layers 1..b -- is committed; on no match everything speculative is
+ * dropped.  Branches are run on every step, the last included, as the paper's compute
+ * count assumes.
+ *
+ * units  : latency in layer time-units with k free extra compute units (paper Section 4.1)
+ * cunits : total compute units (main + branches)
+ */
+int orc_ppd(orc_model* m, int32_t n, int32_t k, int32_t l, int32_t eos, int32_t* tokens,
+            uint8_t* hit, int32_t* n_out, int64_t* units, int64_t* cunits) {
+    const orc_config* c = &m->c;
+    const int D = c->d_model, V = c->vocab, d = c->n_layers;
+    if (m->pending < 0 || n < 0 || k < 1 || k > c->max_k || k > V || l < 1 || l > d) return -1;
+    if (m->pos + n + 1 > c->max_seq) return -2;
+    const int b = l < d - l ? l : d - l;
+    double* h = (double*)malloc(sizeof(double) * D);
+    double* hb = (double*)malloc(sizeof(double) * D * (size_t)k);
+    double* hc = (double*)malloc(sizeof(double) * D);  /* committed hidden state at layer b */
+    double* lg = (double*)malloc(sizeof(double) * V);
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)k);
+    int prev_hit = 0;
+    int64_t u = 0, cu = 0;
+    int s = 0;
+    for (; s < n; ++s) {
+        const int pos = m->pos;
+        if (!prev_hit) {
+            orc_embed(m, m->pending, h);
+            for (int j = 0; j < l; ++j) orc_layer(m, j, h, pos, -1);
+            u += l;
+        } else {
+            memcpy(h, hc, sizeof(double) * D);
+            for (int j = b; j < l; ++j) orc_layer(m, j, h, pos, -1);
+            u += l - b;
+        }
+        orc_head(m, h, lg);
+        orc_topk(lg, V, k, cand);
+        for (int i = 0; i < k; ++i) {
+            double* hi = hb + (size_t)i * D;
+            orc_embed(m, cand[i], hi);
+            for (int j = 0; j < b; ++j) orc_layer(m, j, hi, pos + 1, i);
+        }
+        cu += (int64_t)k * b;
+        for (int j = l; j < d; ++j) orc_layer(m, j, h, pos, -1);
+        u += d - l;
+        orc_head(m, h, lg);
+        int32_t next;
+        orc_topk(lg, V, 1, &next);
+        int istar = -1;
+        for (int i = 0; i < k; ++i) if (cand[i] == next) istar = i;
+        if (istar >= 0) {
+            for (int j = 0; j < b; ++j) {
+                size_t src = ((size_t)istar * c->n_layers + j) * D;
+                size_t dst = ((size_t)j * c->max_seq + (size_t)(pos + 1)) * D;
+                memcpy(m->kc + dst, m->kb + src, sizeof(double) * D);
+                memcpy(m->vc + dst, m->vb + src, sizeof(double) * D);
+            }
+            memcpy(hc, hb + (size_t)istar * D, sizeof(double) * D);
+        }
+        prev_hit = istar >= 0;
+        tokens[s] = next;
+        hit[s] = (uint8_t)prev_hit;
+        m->pending = next;
+        m->pos = pos + 1;
+        if (eos >= 0 && next == eos) { ++s; break; }
+    }
+    cu += u;
+    if (n_out) *n_out = s;
+    if (units) *units = u;
+    if (cunits) *cunits = cu;
+    free(h); free(hb); free(hc); free(lg); free(cand);
+    return 0;
+}

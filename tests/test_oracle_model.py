@@ -1,0 +1,217 @@
+"""Pins for the oracle's transformer: an independent float64 PyTorch composition of library
+routines (full recompute, no cache), the Hugging Face LLaMA module on the same blob, and
+invariants of the individual pieces."""
+import math
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import oracle
+import ppd_inputs
+from oracle import Oracle
+
+SMALL = ppd_inputs.ModelShape("small", n_layers=3, d_model=64, n_heads=4, head_dim=16, d_ffn=176, vocab=512)
+
+
+def _t(a):
+    return torch.from_numpy(ppd_inputs.bf16_to_f32(np.asarray(a))).double()
+
+
+def bf16_round_f64(x):
+    """Round float64 to 7 mantissa bits (ties to even) in one step by integer arithmetic on the
+    bit pattern; valid for magnitudes in the normal bf16 range."""
+    bits = x.contiguous().view(torch.int64)
+    bits = bits + ((1 << 44) - 1) + ((bits >> 45) & 1)
+    return (bits & ~((1 << 45) - 1)).view(torch.float64)
+
+
+def torch_full_forward(shape, blob, tokens, kv_round):
+    """Logits [T][V] and per-layer hidden states, recomputed from scratch for the whole sequence."""
+    w = ppd_inputs.blob_views(shape, blob)
+    T, D, H, hd = len(tokens), shape.d_model, shape.n_heads, shape.head_dim
+    h = _t(w["E"])[torch.as_tensor(tokens, dtype=torch.long)]
+    pos = torch.arange(T, dtype=torch.float64)
+    inv_freq = shape.rope_theta ** (-torch.arange(0, hd, 2, dtype=torch.float64) / hd)
+    ang = pos[:, None] * inv_freq[None, :]
+    cos, sin = torch.cat([ang.cos(), ang.cos()], -1), torch.cat([ang.sin(), ang.sin()], -1)
+
+    def rot(x):  # [H, T, hd]
+        x1, x2 = x[..., : hd // 2], x[..., hd // 2:]
+        return x * cos + torch.cat([-x2, x1], -1) * sin
+
+    hidden = [h.clone()]
+    for i in range(shape.n_layers):
+        n = F.rms_norm(h, (D,), weight=_t(w[f"g1.{i}"]), eps=shape.rms_eps)
+        q = (n @ _t(w[f"Wq.{i}"]).T).view(T, H, hd).transpose(0, 1)
+        k = (n @ _t(w[f"Wk.{i}"]).T).view(T, H, hd).transpose(0, 1)
+        v = (n @ _t(w[f"Wv.{i}"]).T).view(T, H, hd).transpose(0, 1)
+        q, k = rot(q), rot(k)
+        if kv_round:
+            k, v = bf16_round_f64(k), bf16_round_f64(v)
+        a = F.scaled_dot_product_attention(q[None], k[None], v[None], is_causal=True)[0]
+        h = h + a.transpose(0, 1).reshape(T, D) @ _t(w[f"Wo.{i}"]).T
+        n = F.rms_norm(h, (D,), weight=_t(w[f"g2.{i}"]), eps=shape.rms_eps)
+        z = F.silu(n @ _t(w[f"Wg.{i}"]).T) * (n @ _t(w[f"Wu.{i}"]).T)
+        h = h + z @ _t(w[f"Wd.{i}"]).T
+        hidden.append(h.clone())
+    logits = F.rms_norm(h, (D,), weight=_t(w["g_final"]), eps=shape.rms_eps) @ _t(w["W_H"]).T
+    return logits.numpy(), hidden
+
+
+def oracle_teacher_forced(shape, blob, tokens, kv_round, k=0, l=1):
+    """Incremental (cached) oracle logits for every position of a given token sequence."""
+    o = Oracle(shape, blob, max_seq=len(tokens) + 2, kv_round_bf16=kv_round)
+    o.prefill(tokens[:1])
+    forced = list(tokens[1:]) + [0]
+    r = o.greedy_probe(len(tokens), k=k, l=l, forced=forced, dump_logits=True)
+    o.close()
+    return r
+
+
+@pytest.mark.parametrize("kv_round,tol", [(False, 1e-10), (True, 1e-6)])
+@pytest.mark.parametrize("resid_scale", [0.1, 1.0])
+def test_logits_match_float64_torch_composition(kv_round, tol, resid_scale):
+    blob = ppd_inputs.gen_weights(SMALL, seed=3, resid_scale=resid_scale, sigma=0.08)
+    tokens = ppd_inputs.gen_prompt(SMALL.vocab, 21, seed=4)
+    ref, _ = torch_full_forward(SMALL, blob, tokens, kv_round)
+    got = oracle_teacher_forced(SMALL, blob, tokens, kv_round)["final_logits"]
+    assert np.abs(ref).max() > 0.05            # the comparison is not vacuous
+    assert np.abs(got - ref).max() < tol
+
+
+def test_tiny_config_logits_and_early_head(tiny_shape, tiny_blob, tiny_prompt):
+    # early logits after layer l = W_H . RMSNorm_final(hidden state after l blocks)
+    l = 2
+    ref, hidden = torch_full_forward(tiny_shape, tiny_blob, tiny_prompt, True)
+    w = ppd_inputs.blob_views(tiny_shape, tiny_blob)
+    early_ref = (F.rms_norm(hidden[l], (tiny_shape.d_model,), weight=_t(w["g_final"]), eps=tiny_shape.rms_eps)
+                 @ _t(w["W_H"]).T).numpy()
+    r = oracle_teacher_forced(tiny_shape, tiny_blob, tiny_prompt, True, k=3, l=l)
+    assert np.abs(r["final_logits"] - ref).max() < 1e-6
+    assert np.abs(r["early_logits"] - early_ref).max() < 1e-6
+    # argmax / top-k / hit definitions against numpy on the reference logits
+    order = np.lexsort((np.arange(tiny_shape.vocab)[None, :].repeat(len(tiny_prompt), 0), -ref), axis=-1)
+    assert (r["tokens"] == order[:, 0]).all()
+    e_order = np.lexsort((np.arange(tiny_shape.vocab)[None, :].repeat(len(tiny_prompt), 0), -early_ref), axis=-1)
+    assert (r["cand"] == e_order[:, :3]).all()
+    assert (r["hit"] == [(t in c) for t, c in zip(r["tokens"], r["cand"])]).all()
+    srt = -np.sort(-ref, axis=-1)
+    assert np.allclose(r["margin_final"], srt[:, 0] - srt[:, 1], atol=1e-6)
+
+
+def test_against_huggingface_llama():
+    transformers = pytest.importorskip("transformers")
+    shape = SMALL
+    blob = ppd_inputs.gen_weights(shape, seed=5, sigma=0.08, resid_scale=0.5)
+    tokens = ppd_inputs.gen_prompt(shape.vocab, 17, seed=6)
+    kw = dict(hidden_size=shape.d_model, intermediate_size=shape.d_ffn, num_hidden_layers=shape.n_layers,
+              num_attention_heads=shape.n_heads, num_key_value_heads=shape.n_heads, vocab_size=shape.vocab,
+              rms_norm_eps=shape.rms_eps, max_position_embeddings=64, attention_bias=False, mlp_bias=False,
+              tie_word_embeddings=False, hidden_act="silu")
+    try:
+        cfg = transformers.LlamaConfig(rope_theta=shape.rope_theta, **kw)
+    except TypeError:
+        cfg = transformers.LlamaConfig(rope_parameters={"rope_type": "default", "rope_theta": shape.rope_theta}, **kw)
+    cfg._attn_implementation = "eager"
+    model = transformers.LlamaForCausalLM(cfg).double().eval()
+    w = ppd_inputs.blob_views(shape, blob)
+    sd = {"model.embed_tokens.weight": _t(w["E"]), "model.norm.weight": _t(w["g_final"]),
+          "lm_head.weight": _t(w["W_H"])}
+    names = {"Wq": "self_attn.q_proj", "Wk": "self_attn.k_proj", "Wv": "self_attn.v_proj",
+             "Wo": "self_attn.o_proj", "Wg": "mlp.gate_proj", "Wu": "mlp.up_proj", "Wd": "mlp.down_proj",
+             "g1": "input_layernorm", "g2": "post_attention_layernorm"}
+    for i in range(shape.n_layers):
+        for ours, theirs in names.items():
+            sd[f"model.layers.{i}.{theirs}.weight"] = _t(w[f"{ours}.{i}"])
+    missing, unexpected = model.load_state_dict(sd, strict=False)
+    assert not [m for m in missing if "rotary" not in m] and not unexpected
+    with torch.no_grad():
+        ref = model(torch.as_tensor(tokens, dtype=torch.long)[None]).logits[0].numpy()
+    got = oracle_teacher_forced(shape, blob, tokens, False)["final_logits"]
+    assert np.abs(ref).max() > 0.05
+    # the library keeps float32 internals (norm variance, rotary tables) even in a float64 model, so
+    # agreement is at float32 level; a wrong convention (rotary pairing, norm, scale) is off by > 1e-2
+    assert np.abs(got - ref).max() < 5e-6
+
+
+def test_rmsnorm_unit_rms_and_scale_invariance():
+    rng = np.random.default_rng(0)
+    h = rng.standard_normal(256) * 3.0
+    ones = np.full(256, 0x3F80, dtype=np.uint16)
+    out = oracle.rmsnorm(h, ones, 0.0)
+    assert abs(np.sqrt(np.mean(out ** 2)) - 1.0) < 1e-12
+    assert np.allclose(oracle.rmsnorm(7.5 * h, ones, 0.0), out, atol=1e-12)
+    g = ppd_inputs.gen_weights(SMALL, seed=9)[:256]
+    assert np.allclose(oracle.rmsnorm(h, g, 1e-5),
+                       ppd_inputs.bf16_to_f32(g) * h / np.sqrt(np.mean(h ** 2) + 1e-5), atol=1e-12)
+
+
+def test_rope_is_a_rotation_by_relative_position():
+    rng = np.random.default_rng(1)
+    H, hd, theta = 2, 16, 10000.0
+    q, k = rng.standard_normal(H * hd), rng.standard_normal(H * hd)
+    base = oracle.rope(q, H, hd, 5, theta) @ oracle.rope(k, H, hd, 2, theta)
+    for shift in (1, 7, 100):
+        assert abs(oracle.rope(q, H, hd, 5 + shift, theta) @ oracle.rope(k, H, hd, 2 + shift, theta) - base) < 1e-9
+    assert np.allclose(oracle.rope(q, H, hd, 0, theta), q)                      # position 0: identity
+    assert abs(np.linalg.norm(oracle.rope(q, H, hd, 31, theta)) - np.linalg.norm(q)) < 1e-12
+    # pair (i, i + hd/2) turns by pos * theta^(-2i/hd): check one pair by hand
+    r = oracle.rope(q, H, hd, 3, theta)
+    i = 2
+    ang = 3 * theta ** (-2 * i / hd)
+    assert abs(r[i] - (q[i] * math.cos(ang) - q[i + hd // 2] * math.sin(ang))) < 1e-12
+    assert abs(r[i + hd // 2] - (q[i + hd // 2] * math.cos(ang) + q[i] * math.sin(ang))) < 1e-12
+
+
+def test_attention_special_cases():
+    rng = np.random.default_rng(2)
+    H, hd = 2, 8
+    D = H * hd
+    q = rng.standard_normal(D)
+    kc, vc = rng.standard_normal((5, D)), rng.standard_normal((5, D))
+    # one position: output is that position's value
+    assert np.allclose(oracle.attention(q, kc[:1], vc[:1], n_heads=H, head_dim=hd), vc[0])
+    # zero query: uniform average of the values
+    assert np.allclose(oracle.attention(np.zeros(D), kc, vc, n_heads=H, head_dim=hd), vc.mean(0))
+    # a tail position is the same as one more canonical row
+    a = oracle.attention(q, kc, vc, n_heads=H, head_dim=hd)
+    b = oracle.attention(q, kc[:4], vc[:4], kc[4], vc[4], n_heads=H, head_dim=hd)
+    assert np.allclose(a, b, atol=1e-14)
+    # library softmax
+    ref = np.empty(D)
+    for h in range(H):
+        s = torch.softmax(torch.from_numpy(kc[:, h * hd:(h + 1) * hd] @ q[h * hd:(h + 1) * hd] / math.sqrt(hd)), 0)
+        ref[h * hd:(h + 1) * hd] = s.numpy() @ vc[:, h * hd:(h + 1) * hd]
+    assert np.allclose(a, ref, atol=1e-13)
+
+
+def test_silu_and_matvec():
+    assert oracle.silu(0.0) == 0.0
+    assert abs(oracle.silu(2.0) - 2.0 / (1 + math.exp(-2.0))) < 1e-15
+    assert abs(oracle.silu(-30.0)) < 1e-11
+    rng = np.random.default_rng(3)
+    w = ppd_inputs.gen_weights(SMALL, seed=2)[: 24 * 40].reshape(24, 40)
+    x = rng.standard_normal(40)
+    assert np.allclose(oracle.matvec(w, x), ppd_inputs.bf16_to_f32(w).astype(np.float64) @ x, atol=1e-14)
+    # a transposed operand would fail this: non-square with distinct rows
+    assert not np.allclose(oracle.matvec(w, x)[:5], (ppd_inputs.bf16_to_f32(w).astype(np.float64).T[:5, :24] @ x[:24]))
+
+
+def test_bf16_rounding_matches_library_and_ties_to_even():
+    xs = np.array([1.0, 1.00390625, 1.001953125, 1.005859375, -3.1415926, 1e-3, 65504.0, 2.0 ** -130, 0.0])
+    ref = torch.from_numpy(xs).float().bfloat16().double().numpy()
+    assert (oracle.round_bf16(xs) == ref).all()
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7: even mantissa wins (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    assert oracle.round_bf16(1.00390625) == 1.0
+    assert oracle.round_bf16(1.01171875) == 1.015625
+
+
+def test_topk_order_and_ties():
+    rng = np.random.default_rng(4)
+    lg = rng.standard_normal(97)
+    assert (oracle.topk(lg, 8) == np.argsort(-lg, kind="stable")[:8]).all()
+    tied = np.array([0.5, 2.0, 2.0, -1.0, 2.0, 0.5])
+    assert list(oracle.topk(tied, 5)) == [1, 2, 4, 0, 5]     # value descending, id ascending
+    assert list(oracle.topk(np.zeros(4), 4)) == [0, 1, 2, 3]

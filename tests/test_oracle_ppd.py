@@ -1,0 +1,126 @@
+"""Pins for the oracle's PPD state machine: exactness (PPD tokens == greedy tokens), the
+definition of a match, special cases, and the unit accounting of Theorem 4.1."""
+import numpy as np
+import pytest
+
+import ppd_inputs
+from oracle import Oracle, theory
+
+TOY = ppd_inputs.ModelShape("toy", n_layers=6, d_model=32, n_heads=2, head_dim=16, d_ffn=80, vocab=64)
+
+
+def run_both(shape, blob, prompt, n, k, l, **kw):
+    o = Oracle(shape, blob, max_seq=len(prompt) + n + 2, max_k=max(k, 1), **kw)
+    o.prefill(prompt)
+    g = o.greedy_probe(n, k=k, l=l)
+    o.prefill(prompt)
+    p = o.ppd(n, k, l)
+    o.close()
+    return g, p
+
+
+def test_exactness_all_k_and_layers_tiny(tiny_shape, tiny_blob, tiny_prompt):
+    d, n = tiny_shape.n_layers, 12
+    hits_seen = set()
+    for l in range(1, d):
+        for k in range(1, 9):
+            g, p = run_both(tiny_shape, tiny_blob, tiny_prompt, n, k, l)
+            assert (p["tokens"] == g["tokens"]).all(), (k, l)
+            assert (p["hit"] == g["hit"]).all(), (k, l)
+            lat, cmp_ = theory.realised_units(d, l, k, list(g["hit"]))
+            assert (p["units"], p["cunits"]) == (lat, cmp_)
+            b = theory.branch_depth(d, l)
+            assert p["units"] == d * n - b * int(g["hit"][:-1].sum())          # Theorem 4.1, realised count
+            assert p["cunits"] == p["units"] + k * b * n
+            hits_seen.update(g["hit"].tolist())
+    assert hits_seen == {0, 1}       # both the commit and the discard paths were exercised
+
+
+def test_tiny_workload_config(tiny_shape, tiny_blob, tiny_prompt):
+    # the small benchmark configuration: prompt 16, generate 32, k = 3 at layer 2
+    g, p = run_both(tiny_shape, tiny_blob, tiny_prompt, 32, 3, 2)
+    assert (p["tokens"] == g["tokens"]).all() and (p["hit"] == g["hit"]).all()
+    assert 0 < g["hit"].mean() < 1
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_exactness_toy_with_commit_chains(seed):
+    # weak residual branches: early predictions mostly agree, so long runs of consecutive commits
+    blob = ppd_inputs.gen_weights(TOY, seed=seed, sigma=0.3, resid_scale=0.03)
+    prompt = ppd_inputs.gen_prompt(TOY.vocab, 5, seed=seed + 1)
+    for l in (2, 3, 4, 5):
+        g, p = run_both(TOY, blob, prompt, 24, 2, l)
+        assert (p["tokens"] == g["tokens"]).all() and (p["hit"] == g["hit"]).all()
+    assert g["hit"].mean() > 0.5
+
+
+def test_early_layer_equal_to_depth_always_hits():
+    blob = ppd_inputs.gen_weights(TOY, seed=2, sigma=0.3)
+    prompt = ppd_inputs.gen_prompt(TOY.vocab, 4, seed=3)
+    g, p = run_both(TOY, blob, prompt, 10, 1, TOY.n_layers)
+    assert g["hit"].all() and p["hit"].all() and (p["tokens"] == g["tokens"]).all()
+    assert p["units"] == TOY.n_layers * 10      # b = 0: nothing is saved
+
+
+def test_k_equal_vocab_always_hits():
+    blob = ppd_inputs.gen_weights(TOY, seed=4, sigma=0.3, resid_scale=1.0)
+    prompt = ppd_inputs.gen_prompt(TOY.vocab, 4, seed=5)
+    o = Oracle(TOY, blob, max_seq=32, max_k=TOY.vocab)
+    o.prefill(prompt)
+    g = o.greedy_probe(8, k=TOY.vocab, l=3)
+    o.prefill(prompt)
+    p = o.ppd(8, TOY.vocab, 3)
+    assert g["hit"].all() and p["hit"].all() and (p["tokens"] == g["tokens"]).all()
+    assert p["units"] == 6 * 8 - 3 * 7
+
+
+def test_k1_hits_iff_early_argmax_equals_final_argmax():
+    blob = ppd_inputs.gen_weights(TOY, seed=6, sigma=0.3, resid_scale=0.2)
+    prompt = ppd_inputs.gen_prompt(TOY.vocab, 6, seed=7)
+    o = Oracle(TOY, blob, max_seq=40)
+    o.prefill(prompt)
+    g = o.greedy_probe(20, k=1, l=4, dump_logits=True)
+    assert (g["hit"] == (g["early_logits"].argmax(1) == g["final_logits"].argmax(1))).all()
+    assert 0 < g["hit"].sum() < 20
+
+
+def test_eos_stops_after_emitting_it(tiny_shape, tiny_blob, tiny_prompt):
+    o = Oracle(tiny_shape, tiny_blob, max_seq=64)
+    o.prefill(tiny_prompt)
+    ref = o.ppd(10, 3, 2)["tokens"]
+    o.prefill(tiny_prompt)
+    cut = o.ppd(10, 3, 2, eos=int(ref[4]))["tokens"]
+    first = int(np.argmax(ref == ref[4]))
+    assert (cut == ref[: first + 1]).all()
+
+
+def test_greedy_continues_identically_after_ppd(tiny_shape, tiny_blob, tiny_prompt):
+    # committed cache state after PPD equals the greedy cache: continuing either way gives one stream
+    o = Oracle(tiny_shape, tiny_blob, max_seq=64)
+    o.prefill(tiny_prompt)
+    a = np.concatenate([o.ppd(7, 3, 2)["tokens"], o.greedy_probe(7)["tokens"], o.ppd(6, 2, 3)["tokens"]])
+    o.prefill(tiny_prompt)
+    assert (a == o.greedy_probe(20)["tokens"]).all()
+
+
+def test_kv_rounding_switch_changes_little(tiny_shape, tiny_blob, tiny_prompt):
+    outs = []
+    for kv in (True, False):
+        o = Oracle(tiny_shape, tiny_blob, max_seq=64, kv_round_bf16=kv)
+        o.prefill(tiny_prompt)
+        outs.append(o.greedy_probe(4, dump_logits=True)["final_logits"])
+    diff = np.abs(outs[0] - outs[1]).max()
+    assert 0 < diff < 5e-3
+
+
+def test_argument_checks(tiny_shape, tiny_blob, tiny_prompt):
+    o = Oracle(tiny_shape, tiny_blob, max_seq=24, max_k=4)
+    with pytest.raises(ValueError):
+        o.ppd(4, 3, 2)                       # before prefill
+    o.prefill(tiny_prompt)
+    with pytest.raises(ValueError):
+        o.ppd(4, 5, 2)                       # k > max_k
+    with pytest.raises(ValueError):
+        o.ppd(4, 3, 0)                       # early layer out of range
+    with pytest.raises(ValueError):
+        o.ppd(20, 3, 2)                      # cache would overflow
