@@ -1,0 +1,199 @@
+/*
+ * ppd.h -- C ABI of the B200 (sm_100a) Predictive Pipelined Decoding library.
+ *
+ * PPD (Yang et al., "Predictive Pipelined Decoding: A Compute-Latency Trade-off for Exact
+ * LLM Decoding", Section 3, Algorithms 1 and 2) is exact greedy decoding in which, while the
+ * main pass of the current token finishes layers l+1..d, the top-k tokens predicted by an
+ * early head after layer l already start their own forward passes; the final argmax then
+ * verifies the candidates and the matching branch is kept.  The token stream equals plain
+ * greedy decoding.
+ *
+ * Conventions
+ *   - Model: decoder-only transformer with RMSNorm, rotate-half RoPE (dims i and i+hd/2
+ *     paired, angle pos * theta^(-2i/hd)), multi-head causal attention (n_heads * head_dim
+ *     == d_model), SwiGLU FFN, untied unembedding W_H; no biases.
+ *   - The early head is the final head applied to the hidden state after l blocks:
+ *     W_H . RMSNorm_final(h_l)   (the untrained-classifier variant, Table 2 column "N").
+ *   - Top-k / argmax order: logit descending, token id ascending.
+ *   - b = min(l, d - l) layers are run by each candidate branch before verification
+ *     (the paper's d - l for l >= d/2).
+ *   - "host" / "device" is stated for every pointer.  All functions return 0 on success or a
+ *     negative PPD_E* code; none throws, aborts or allocates device memory.  Unless stated
+ *     otherwise a call is synchronous: its work has finished when it returns.
+ *   - One ppd_ctx must be used from one host thread at a time.
+ */
+#ifndef PPD_H
+#define PPD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PPD_OK 0
+#define PPD_EINVAL (-1)   /* bad argument or shape                                   */
+#define PPD_ENOSPC (-2)   /* KV cache (max_seq) or device arena too small           */
+#define PPD_ESTATE (-3)   /* call out of order (decode before load/prefill)         */
+#define PPD_ECUDA (-4)    /* a CUDA call failed; see ppd_last_cuda_error            */
+#define PPD_ETIMEOUT (-5) /* a bounded device-side wait gave up; outputs are invalid */
+
+#define PPD_MAX_K 8       /* largest supported number of early candidates            */
+
+typedef struct ppd_ctx ppd_ctx;
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t max_seq;        /* KV capacity in positions (prompt + generated + 1)      */
+    int32_t max_k;          /* 0..PPD_MAX_K branch slots                              */
+    int32_t kv_page_tokens; /* positions per KV page; must be 64                      */
+    float rms_eps, rope_theta;
+} ppd_config;
+
+typedef struct {
+    int64_t steps;          /* decode steps executed since create/reset_stats        */
+    int64_t hits;           /* of which the early candidates contained the token     */
+    int64_t steps_after_hit;/* steps whose main pass started at layer b              */
+    int64_t kernel_launches;/* kernels of this library launched by decode steps      */
+    double ms_decode;       /* device time of the last ppd_decode / greedy loop (ms) */
+    double ms_steps_fresh;  /* summed device time of steps that followed a miss      */
+    double ms_steps_cont;   /* summed device time of steps that followed a hit       */
+} ppd_stats;
+
+/* ---------------------------------------------------------------- context */
+
+/* Bytes of device memory a context needs (packed weights, KV pages, branch slots, workspace).
+ * Returns 0 for an invalid config.  cfg: host. */
+size_t ppd_device_bytes(const ppd_config* cfg);
+
+/* Creates a context inside caller-owned device memory.
+ * dev_mem: device, >= ppd_device_bytes(cfg) bytes, 256-byte aligned; owned by the caller and
+ * kept alive (and untouched) until ppd_destroy.  stream_main / stream_branch: cudaStream_t
+ * handles owned by the caller, distinct, on the current device.  *out: host. */
+int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes,
+               void* stream_main, void* stream_branch, ppd_ctx** out);
+void ppd_destroy(ppd_ctx* ctx);
+
+/* Uploads the weights and converts them to the device layout (bf16 tiles, fused Wq|Wk|Wv and
+ * row-interleaved Wg/Wu).  host_blob: host, may be freed on return.  Tensor order, all
+ * row-major [out][in]:  E[V][D]; per layer g1[D] Wq Wk Wv Wo [D][D] g2[D] Wg Wu [F][D] Wd[D][F];
+ * g_final[D]; W_H[V][D].  dtype: 1 = bf16 (uint16 bit patterns), 0 = float32 (rounded to bf16,
+ * nearest-even).  bytes must equal the blob size for cfg. */
+int ppd_load_weights(ppd_ctx* ctx, const void* host_blob, size_t bytes, int dtype);
+
+/* ---------------------------------------------------------------- decoding */
+
+/* Fills the KV cache from a prompt (host, n_prompt >= 1 ids in [0, vocab)).  The last prompt
+ * token is the start token x_0 of Algorithm 1: positions 0..n_prompt-2 are cached and
+ * prompt[n_prompt-1] stays pending for the first decode step.  Resets the position. */
+int ppd_prefill(ppd_ctx* ctx, const int32_t* prompt, int32_t n_prompt);
+
+/* One conventional greedy step: all d layers, argmax of the final logits (Section 1).
+ * out_token: host, one id. */
+int ppd_greedy_step(ppd_ctx* ctx, int32_t* out_token);
+
+/* Generates up to n_tokens tokens.  k = 0: plain greedy loop.  k >= 1: PPD with k candidates
+ * from the early head after layer l (1 <= l <= d-1), Algorithm 2.  eos = -1 disables the stop
+ * token; otherwise generation stops after emitting eos.
+ * out_tokens [n_tokens], out_hit [n_tokens], out_n [1]: host.  out_hit[s] = 1 iff the final
+ * argmax of step s was among that step's k early candidates (Table 2's match).  Nothing beyond
+ * index *out_n is written.  The tokens equal those of ppd_greedy_step from the same state. */
+int ppd_decode(ppd_ctx* ctx, int32_t k, int32_t l, int32_t n_tokens, int32_t eos,
+               int32_t* out_tokens, uint8_t* out_hit, int32_t* out_n);
+
+/* One PPD step with the host in the loop: the token to feed comes from host memory (pinned or
+ * not) and the result is copied back before returning.  in_token: host, one id, or NULL to
+ * continue with the pending token.  Feeding a token other than the pending one discards any
+ * committed branch.  out_token, out_hit: host. */
+int ppd_step(ppd_ctx* ctx, int32_t k, int32_t l, const int32_t* in_token,
+             int32_t* out_token, uint8_t* out_hit);
+
+/* Drops cached positions >= pos and makes `pending_token` the token to feed at position pos
+ * (re-timing from the end of the prompt: pos = n_prompt-1, pending_token = prompt[n_prompt-1]). */
+int ppd_rewind(ppd_ctx* ctx, int32_t pos, int32_t pending_token);
+
+/* Position of the pending token (= number of cached positions). */
+int32_t ppd_position(const ppd_ctx* ctx);
+
+/* ---------------------------------------------------------------- inspection */
+
+int ppd_get_stats(ppd_ctx* ctx, ppd_stats* out);   /* out: host */
+int ppd_reset_stats(ppd_ctx* ctx);
+
+/* Logits of the most recent step: final_logits [vocab], early_logits [vocab] (either may be
+ * NULL): host, float32.  early_logits are those of the last PPD step's early head. */
+int ppd_debug_logits(ppd_ctx* ctx, float* final_logits, float* early_logits);
+/* Top-1 minus top-2 of the last step's final logits, and the k early candidates of the last
+ * PPD step (cand: host [k] or NULL). */
+int ppd_debug_last(ppd_ctx* ctx, float* final_margin, int32_t* cand, int32_t k);
+/* Replaces the pending token (teacher forcing for parity runs); drops any committed branch. */
+int ppd_debug_force_token(ppd_ctx* ctx, int32_t token);
+/* Applies a permutation to the KV page table (host, n_pages entries, a permutation of
+ * 0..n_pages-1, n_pages = ceil(max_seq / kv_page_tokens)); only valid right after create or
+ * before prefill.  Exists to test that kernels honour the page table. */
+int ppd_debug_set_page_table(ppd_ctx* ctx, const int32_t* table, int32_t n_pages);
+
+const char* ppd_strerror(int code);
+/* Text of the last CUDA error seen by this context (static storage). */
+const char* ppd_last_cuda_error(const ppd_ctx* ctx);
+
+/* ---------------------------------------------------------------- single operations
+ * Stand-alone launches of the hot-path kernels on caller-owned device buffers, used by the
+ * kernel-level parity tests and benchmarks.  `stream` is a cudaStream_t handle (NULL = default
+ * stream).  These calls only enqueue work; the caller synchronises.                          */
+
+/* Bytes of the packed form of an [N][K] matrix (32-row x 256-column bf16 tiles). */
+size_t ppd_packed_bytes(int32_t n_rows, int32_t n_cols);
+
+/* Packs rows [0, n_src_rows) of a row-major bf16 matrix src (device, [n_src_rows][n_cols]) into
+ * dst (device, ppd_packed_bytes(n_dst_rows, n_cols), zeroed by the caller for padding).  Source
+ * row r lands in packed row r * row_mul + row_off. */
+int ppd_op_pack(const uint16_t* src, int32_t n_src_rows, int32_t n_cols, void* dst,
+                int32_t n_dst_rows, int32_t row_mul, int32_t row_off, void* stream);
+
+/* Skinny-M matrix product y[m][n] = sum_k W[n][k] x'[m][k], m < M <= 8 (the QKV, O, gate/up,
+ * down and head products of one decoder block for M token rows).
+ *   w_packed: device, packed [N][K].  x: device float32 [M][ldx], ldx a multiple of 256 and
+ *   >= K rounded up to 256, zero beyond K.
+ *   gain: device float32 [K rounded up to 256] or NULL.  If given, x' = RMSNorm(x) with that
+ *   gain and eps (mean over the first K entries); otherwise x' = x.
+ *   mode 0: out[m][n] = y.            out: device float32 [M][ldo]
+ *   mode 1: out[m][n] = resid[m][n] + y   (resid: device [M][ldo]; may alias out)
+ *   mode 2: rows are interleaved gate/up pairs; out[m][j] = silu(y[2j]) * y[2j+1], j < N/2
+ * A row's result does not depend on M or on the other rows. */
+int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
+                const float* gain, float eps, int32_t mode, const float* resid, float* out,
+                int32_t ldo, void* stream);
+
+/* Head: logits[m][v] = W_H . RMSNorm(x[m]) for M rows and the k largest per row in the order
+ * (value descending, id ascending).  scratch: device, >= ppd_op_head_scratch_bytes() bytes,
+ * zeroed once by the caller before first use (the kernel leaves it zeroed).
+ * logits: device float32 [M][vocab]; top_ids: device int32 [M][k]; top_vals: device float32 [M][k]. */
+size_t ppd_op_head_scratch_bytes(void);
+int ppd_op_head_topk(const void* w_packed, int32_t vocab, int32_t K, const float* x, int32_t M,
+                     int32_t ldx, const float* gain, float eps, int32_t k, void* scratch,
+                     float* logits, int32_t* top_ids, float* top_vals, void* stream);
+
+/* Decode attention for M query rows that share a cached prefix (Section 3: every process is fed
+ * the same history x_<=t plus its own candidate).
+ *   qkv: device float32 [M][3*D] un-rotated q|k|v of the M new tokens, all at position n_prefix.
+ *   kv_pages: device bf16, one layer's pages; page p holds [2 (K,V)][H][64][hd]; page_table:
+ *   device int32, logical page -> physical page.
+ *   Row m attends to cached positions 0..n_prefix-1 and to its own new K/V.  The rotated,
+ *   bf16-rounded K/V of row m is written to branch_slots + m*2*D (device bf16 [M][2][H][hd]) or,
+ *   when branch_slots is NULL, into the cache at position n_prefix (main pass; M = 1).
+ *   rope_table: device float2 [>= n_prefix+1][hd/2] (cos, sin) as made by ppd_op_rope_table.
+ *   scratch: device, >= ppd_op_attn_scratch_bytes(M, H, hd, n_prefix+1) bytes, zeroed once by the
+ *   caller (the kernel leaves its counters zeroed).  out: device float32 [M][ldo].
+ * A row's result does not depend on M or on the other rows. */
+size_t ppd_op_attn_scratch_bytes(int32_t M, int32_t n_heads, int32_t head_dim, int32_t n_positions);
+int ppd_op_rope_table(float* table, int32_t n_positions, int32_t head_dim, float theta, void* stream);
+int ppd_op_attention(const float* qkv, int32_t M, int32_t n_heads, int32_t head_dim, int32_t n_prefix,
+                     void* kv_pages, const int32_t* page_table, void* branch_slots,
+                     const float* rope_table, void* scratch, float* out, int32_t ldo, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PPD_H */

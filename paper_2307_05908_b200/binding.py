@@ -1,0 +1,265 @@
+"""Thin ctypes binding of libppd_b200.so: argument marshalling only.
+
+PyTorch supplies device memory and streams; every step of the decode path runs in the CUDA
+library.  There is no CPU fallback: if the library is missing or a call fails, an exception is
+raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_LIB = None
+
+PPD_MAX_K = 8
+ERRORS = {0: "PPD_OK", -1: "PPD_EINVAL", -2: "PPD_ENOSPC", -3: "PPD_ESTATE", -4: "PPD_ECUDA", -5: "PPD_ETIMEOUT"}
+
+
+class PPDError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"{ERRORS.get(code, code)}: {text}")
+        self.code = code
+
+
+class Config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab", "max_seq", "max_k",
+                 "kv_page_tokens")] + [("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("steps", ctypes.c_int64), ("hits", ctypes.c_int64), ("steps_after_hit", ctypes.c_int64),
+                ("kernel_launches", ctypes.c_int64), ("ms_decode", ctypes.c_double),
+                ("ms_steps_fresh", ctypes.c_double), ("ms_steps_cont", ctypes.c_double)]
+
+
+_P, _I, _F, _SZ = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+_CFG = ctypes.POINTER(Config)
+
+# every symbol include/ppd.h declares: name -> (restype, argtypes)
+SIGNATURES = {
+    "ppd_device_bytes": (_SZ, [_CFG]),
+    "ppd_create": (ctypes.c_int, [_CFG, _P, _SZ, _P, _P, ctypes.POINTER(_P)]),
+    "ppd_destroy": (None, [_P]),
+    "ppd_load_weights": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int]),
+    "ppd_prefill": (ctypes.c_int, [_P, _P, _I]),
+    "ppd_greedy_step": (ctypes.c_int, [_P, _P]),
+    "ppd_decode": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P]),
+    "ppd_step": (ctypes.c_int, [_P, _I, _I, _P, _P, _P]),
+    "ppd_rewind": (ctypes.c_int, [_P, _I, _I]),
+    "ppd_position": (_I, [_P]),
+    "ppd_get_stats": (ctypes.c_int, [_P, ctypes.POINTER(Stats)]),
+    "ppd_reset_stats": (ctypes.c_int, [_P]),
+    "ppd_debug_logits": (ctypes.c_int, [_P, _P, _P]),
+    "ppd_debug_last": (ctypes.c_int, [_P, _P, _P, _I]),
+    "ppd_debug_force_token": (ctypes.c_int, [_P, _I]),
+    "ppd_debug_set_page_table": (ctypes.c_int, [_P, _P, _I]),
+    "ppd_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "ppd_last_cuda_error": (ctypes.c_char_p, [_P]),
+    "ppd_packed_bytes": (_SZ, [_I, _I]),
+    "ppd_op_pack": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _I, _P]),
+    "ppd_op_gemv": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _I, _P]),
+    "ppd_op_head_scratch_bytes": (_SZ, []),
+    "ppd_op_head_topk": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P, _P]),
+    "ppd_op_attn_scratch_bytes": (_SZ, [_I, _I, _I, _I]),
+    "ppd_op_rope_table": (ctypes.c_int, [_P, _I, _I, _F, _P]),
+    "ppd_op_attention": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _I, _P]),
+}
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Loads the shared library (building it with nvcc first if it is absent or stale)."""
+    global _LIB
+    if _LIB is None:
+        if build_if_missing:
+            _build.build()
+        if not os.path.exists(_build.LIB):
+            raise RuntimeError(f"{_build.LIB} is missing: run paper_2307_05908_b200/build.py (no CPU fallback exists)")
+        lib = ctypes.CDLL(_build.LIB)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _LIB = lib
+    return _LIB
+
+
+def _check(rc, ctx=None):
+    if rc != 0:
+        lib = load()
+        text = lib.ppd_strerror(rc).decode()
+        if rc == -4 and ctx is not None:
+            text += ": " + lib.ppd_last_cuda_error(ctx).decode()
+        raise PPDError(rc, text)
+
+
+def _np_ptr(a):
+    return None if a is None else a.ctypes.data
+
+
+def make_config(shape, max_seq, max_k=PPD_MAX_K) -> Config:
+    return Config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
+                  max_seq, max_k, 64, shape.rms_eps, shape.rope_theta)
+
+
+class Context:
+    """A PPD decoding context.  Device memory and both streams come from torch and are owned here
+    for the lifetime of the context."""
+
+    def __init__(self, shape, max_seq, max_k=PPD_MAX_K, device="cuda:0"):
+        import torch
+        self._torch = torch
+        self.lib = load()
+        self.shape = shape
+        self.cfg = make_config(shape, max_seq, max_k)
+        self.device = torch.device(device)
+        nbytes = self.lib.ppd_device_bytes(ctypes.byref(self.cfg))
+        if nbytes == 0:
+            raise PPDError(-1, "invalid config")
+        self.device_bytes = nbytes
+        with torch.cuda.device(self.device):
+            self.arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            self.stream_main = torch.cuda.Stream(device=self.device)
+            self.stream_branch = torch.cuda.Stream(device=self.device)
+            torch.cuda.synchronize(self.device)
+            base = (self.arena.data_ptr() + 255) // 256 * 256
+            h = _P()
+            _check(self.lib.ppd_create(ctypes.byref(self.cfg), base, nbytes, self.stream_main.cuda_stream,
+                                       self.stream_branch.cuda_stream, ctypes.byref(h)))
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.ppd_destroy(self._h)
+            self._h = None
+            self.arena = None
+
+    __del__ = close
+
+    def _dev(self):
+        return self._torch.cuda.device(self.device)
+
+    def load_weights(self, blob: np.ndarray):
+        """blob: uint16 (bf16 bit patterns) or float32 numpy array in the documented tensor order."""
+        blob = np.ascontiguousarray(blob)
+        dtype = {np.dtype(np.uint16): 1, np.dtype(np.float32): 0}[blob.dtype]
+        with self._dev():
+            _check(self.lib.ppd_load_weights(self._h, blob.ctypes.data, blob.nbytes, dtype), self._h)
+
+    def prefill(self, prompt):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        with self._dev():
+            _check(self.lib.ppd_prefill(self._h, p.ctypes.data, p.size), self._h)
+
+    def greedy_step(self) -> int:
+        out = ctypes.c_int32()
+        with self._dev():
+            _check(self.lib.ppd_greedy_step(self._h, ctypes.byref(out)), self._h)
+        return out.value
+
+    def decode(self, k, l, n_tokens, eos=-1):
+        """Returns (tokens int32[n], hit uint8[n])."""
+        tokens = np.empty(max(n_tokens, 1), dtype=np.int32)
+        hit = np.zeros(max(n_tokens, 1), dtype=np.uint8)
+        n = ctypes.c_int32()
+        with self._dev():
+            _check(self.lib.ppd_decode(self._h, k, l, n_tokens, eos, tokens.ctypes.data, hit.ctypes.data,
+                                       ctypes.byref(n)), self._h)
+        return tokens[: n.value], hit[: n.value]
+
+    def step(self, k, l, in_token=None):
+        """One step with the host in the loop; in_token is a length-1 int32 array (e.g. pinned) or None."""
+        out, hit = ctypes.c_int32(), ctypes.c_uint8()
+        with self._dev():
+            _check(self.lib.ppd_step(self._h, k, l, _np_ptr(in_token), ctypes.byref(out), ctypes.byref(hit)), self._h)
+        return out.value, hit.value
+
+    def rewind(self, pos, pending_token):
+        with self._dev():
+            _check(self.lib.ppd_rewind(self._h, pos, int(pending_token)), self._h)
+
+    @property
+    def position(self):
+        return self.lib.ppd_position(self._h)
+
+    def stats(self) -> Stats:
+        s = Stats()
+        _check(self.lib.ppd_get_stats(self._h, ctypes.byref(s)))
+        return s
+
+    def reset_stats(self):
+        _check(self.lib.ppd_reset_stats(self._h))
+
+    def debug_logits(self, early=False):
+        V = self.shape.vocab
+        fl = np.empty(V, dtype=np.float32)
+        el = np.empty(V, dtype=np.float32) if early else None
+        with self._dev():
+            _check(self.lib.ppd_debug_logits(self._h, fl.ctypes.data, _np_ptr(el)), self._h)
+        return (fl, el) if early else fl
+
+    def debug_last(self, k=0):
+        margin = ctypes.c_float()
+        cand = np.empty(max(k, 1), dtype=np.int32)
+        with self._dev():
+            _check(self.lib.ppd_debug_last(self._h, ctypes.byref(margin), cand.ctypes.data, k), self._h)
+        return margin.value, cand[:k]
+
+    def force_token(self, token):
+        with self._dev():
+            _check(self.lib.ppd_debug_force_token(self._h, int(token)), self._h)
+
+    def set_page_table(self, table):
+        t = np.ascontiguousarray(table, dtype=np.int32)
+        with self._dev():
+            _check(self.lib.ppd_debug_set_page_table(self._h, t.ctypes.data, t.size), self._h)
+
+
+# ------------------------------------------------------------------ single operations on torch tensors
+
+def _s(stream):
+    return None if stream is None else stream.cuda_stream
+
+
+def packed_bytes(n_rows, n_cols) -> int:
+    return load().ppd_packed_bytes(n_rows, n_cols)
+
+
+def op_pack(src, dst, n_dst_rows, row_mul=1, row_off=0, stream=None):
+    """src: torch int16/uint16-viewed bf16 [rows][cols] on device; dst: zeroed uint8 tensor of packed_bytes."""
+    rows, cols = src.shape
+    _check(load().ppd_op_pack(src.data_ptr(), rows, cols, dst.data_ptr(), n_dst_rows, row_mul, row_off, _s(stream)))
+
+
+def op_gemv(w_packed, N, K, x, gain, eps, mode, resid, out, stream=None):
+    M, ldx = x.shape
+    _check(load().ppd_op_gemv(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx,
+                              None if gain is None else gain.data_ptr(), eps, mode,
+                              None if resid is None else resid.data_ptr(), out.data_ptr(), out.shape[1], _s(stream)))
+
+
+def op_head_topk(w_packed, vocab, K, x, gain, eps, k, scratch, logits, top_ids, top_vals, stream=None):
+    M, ldx = x.shape
+    _check(load().ppd_op_head_topk(w_packed.data_ptr(), vocab, K, x.data_ptr(), M, ldx,
+                                   None if gain is None else gain.data_ptr(), eps, k, scratch.data_ptr(),
+                                   logits.data_ptr(), top_ids.data_ptr(), top_vals.data_ptr(), _s(stream)))
+
+
+def op_rope_table(table, n_positions, head_dim, theta, stream=None):
+    _check(load().ppd_op_rope_table(table.data_ptr(), n_positions, head_dim, theta, _s(stream)))
+
+
+def op_attention(qkv, n_heads, head_dim, n_prefix, kv_pages, page_table, branch_slots, rope_table, scratch, out,
+                 stream=None):
+    M = qkv.shape[0]
+    _check(load().ppd_op_attention(qkv.data_ptr(), M, n_heads, head_dim, n_prefix, kv_pages.data_ptr(),
+                                   page_table.data_ptr(), None if branch_slots is None else branch_slots.data_ptr(),
+                                   rope_table.data_ptr(), scratch.data_ptr(), out.data_ptr(), out.shape[1], _s(stream)))

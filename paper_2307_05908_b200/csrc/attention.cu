@@ -1,0 +1,266 @@
+// Decode attention for M query rows over a shared, paged KV prefix (PPD: every candidate branch
+// is fed the same history x_<=t plus its own token, Algorithm 2).
+//
+// All M rows sit at the same position p.  Row m attends to the cached positions 0..p-1, which
+// are read from HBM once for all rows, and to its own new key/value, which it also writes:
+// into the cache (main pass) or into its private branch slot (candidate branch).  RoPE of q and
+// of the new key is applied here, so the QKV product needs no extra pass.
+//
+// Split-KV: split s covers the positions of KV page s.  CTA (head, g) walks the splits
+// s = g, g+G, ...; per split and row it emits (max, sum, weighted V); the last CTA of a head to
+// finish (atomic ticket, no spinning) merges the splits in ascending order.  The split
+// boundaries, the order inside a split and the merge order depend only on positions, never on
+// M or the grid, so a branch row and the main row of the next step get identical bits.
+#include "common.cuh"
+#include "gemv.cuh"
+
+namespace ppd {
+
+constexpr int kAttnThreads = 128;
+constexpr int kAttnWarps = kAttnThreads / 32;
+
+// Rotate-half RoPE of the pair (a, b) = (x_i, x_{i+hd/2}) by (cos, sin); explicit roundings so
+// every instantiation performs the same operations.
+__device__ __forceinline__ float rot_lo(float a, float b, float2 cs) { return __fmaf_rn(a, cs.x, -__fmul_rn(b, cs.y)); }
+__device__ __forceinline__ float rot_hi(float a, float b, float2 cs) { return __fmaf_rn(b, cs.x, __fmul_rn(a, cs.y)); }
+
+template <int HD>
+struct AttnSmem {
+    static constexpr int kTile = kPageTokens * HD * 2;                 // one K or V tile, bytes
+    static constexpr int kKOff = 0;
+    static constexpr int kVOff = kTile;
+    static constexpr int kTailOff = 2 * kTile;                         // ktail[8][HD], vtail[8][HD] bf16
+    static constexpr int kQOff = kTailOff + 2 * kMaxRows * HD * 2;     // q[8][HD] f32
+    static constexpr int kScOff = kQOff + kMaxRows * HD * 4;           // sc[8][68] f32
+    static constexpr int kStatOff = kScOff + kMaxRows * 68 * 4;        // (max, sum)[8]
+    static constexpr int kBarOff = kStatOff + kMaxRows * 2 * 4;
+    static constexpr int kBytes = kBarOff + 16;
+};
+
+template <int M, int HD>
+__global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
+    using S = AttnSmem<HD>;
+    constexpr int DPL = HD / 32;  // dims per lane
+    constexpr int HALF = HD / 2;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint16_t* ks = reinterpret_cast<const uint16_t*>(smem + S::kKOff);
+    const uint16_t* vs = reinterpret_cast<const uint16_t*>(smem + S::kVOff);
+    uint16_t* ktail = reinterpret_cast<uint16_t*>(smem + S::kTailOff);
+    uint16_t* vtail = ktail + kMaxRows * HD;
+    float* qs = reinterpret_cast<float*>(smem + S::kQOff);
+    float* sc = reinterpret_cast<float*>(smem + S::kScOff);
+    float* stat = reinterpret_cast<float*>(smem + S::kStatOff);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + S::kBarOff);
+    int* flag = reinterpret_cast<int*>(smem + S::kBarOff + 8);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.x, g = blockIdx.y, G = gridDim.y;
+    const int H = a.H, D = H * HD;
+
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();
+
+    const int p = (a.d_pos ? *a.d_pos : 0) + a.pos_off;  // position of the new tokens = cached positions
+    const int n_splits = p / kPageTokens + 1;
+    const int s_tail = p / kPageTokens;
+    const float sscale = 1.4426950408889634f / sqrtf((float)HD);  // log2(e) / sqrt(hd)
+    const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
+
+    // rotated queries
+    for (int idx = tid; idx < M * HALF; idx += kAttnThreads) {
+        const int m = idx / HALF, i = idx % HALF;
+        const float2 cs = a.rope[(size_t)p * HALF + i];
+        const float q0 = a.qkv[(size_t)m * 3 * D + h * HD + i];
+        const float q1 = a.qkv[(size_t)m * 3 * D + h * HD + i + HALF];
+        qs[m * HD + i] = rot_lo(q0, q1, cs);
+        qs[m * HD + i + HALF] = rot_hi(q0, q1, cs);
+    }
+    // the CTA that owns the tail split rotates, rounds and stores the new key/value of every row
+    const bool owns_tail = (s_tail % G) == g;
+    if (owns_tail) {
+        for (int idx = tid; idx < M * HALF; idx += kAttnThreads) {
+            const int m = idx / HALF, i = idx % HALF;
+            const float2 cs = a.rope[(size_t)p * HALF + i];
+            const float* kr = a.qkv + (size_t)m * 3 * D + D + h * HD;
+            const float* vr = a.qkv + (size_t)m * 3 * D + 2 * D + h * HD;
+            const uint16_t k0 = f32_to_bf16_bits(rot_lo(kr[i], kr[i + HALF], cs));
+            const uint16_t k1 = f32_to_bf16_bits(rot_hi(kr[i], kr[i + HALF], cs));
+            const uint16_t v0 = f32_to_bf16_bits(vr[i]);
+            const uint16_t v1 = f32_to_bf16_bits(vr[i + HALF]);
+            ktail[m * HD + i] = k0; ktail[m * HD + i + HALF] = k1;
+            vtail[m * HD + i] = v0; vtail[m * HD + i + HALF] = v1;
+            uint16_t *kd, *vd;
+            if (a.slots) {
+                kd = a.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                vd = kd + (size_t)H * HD;
+            } else {
+                uint16_t* pg = a.kv_layer + (size_t)a.page_table[s_tail] * page_elems;
+                kd = pg + ((size_t)h * kPageTokens + (p % kPageTokens)) * HD;
+                vd = kd + (size_t)H * kPageTokens * HD;
+            }
+            kd[i] = k0; kd[i + HALF] = k1;
+            vd[i] = v0; vd[i + HALF] = v1;
+        }
+    }
+    __syncthreads();
+
+    float qr[M][DPL];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int j = 0; j < DPL; ++j) qr[m][j] = qs[m * HD + lane * DPL + j];
+
+    uint32_t phase = 0;
+    for (int s = g; s < n_splits; s += G) {
+        const int n_valid = min(kPageTokens, p - s * kPageTokens);  // cached positions in this split
+        const bool tail = (s == s_tail);
+        if (n_valid > 0) {
+            if (tid == 0) {
+                const uint16_t* pg = a.kv_layer + (size_t)a.page_table[s] * page_elems + (size_t)h * kPageTokens * HD;
+                mbar_arrive_expect_tx(bar, 2 * S::kTile);
+                bulk_g2s(smem + S::kKOff, pg, S::kTile, bar);
+                bulk_g2s(smem + S::kVOff, pg + (size_t)H * kPageTokens * HD, S::kTile, bar);
+            }
+            mbar_wait(bar, phase, a.err, kErrKvWait);
+            phase ^= 1;
+        }
+        // scores (in log2 units)
+        for (int t = warp; t < n_valid; t += kAttnWarps) {
+            float kf[DPL];
+            if constexpr (DPL == 4) {
+                const uint2 kk = *reinterpret_cast<const uint2*>(ks + t * HD + lane * 4);
+                kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
+            } else {
+                const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + t * HD + lane * 2);
+                kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
+            }
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                float d = 0.f;
+#pragma unroll
+                for (int j = 0; j < DPL; ++j) d = fmaf(qr[m][j], kf[j], d);
+                d = warp_sum(d);
+                if (lane == 0) sc[m * 68 + t] = d * sscale;
+            }
+        }
+        if (tail) {
+            for (int m = warp; m < M; m += kAttnWarps) {
+                float d = 0.f;
+#pragma unroll
+                for (int j = 0; j < DPL; ++j) d = fmaf(qr[m][j], bf16_bits_to_f32(ktail[m * HD + lane * DPL + j]), d);
+                d = warp_sum(d);
+                if (lane == 0) sc[m * 68 + n_valid] = d * sscale;
+            }
+        }
+        __syncthreads();
+        const int cnt = n_valid + (tail ? 1 : 0);  // <= 64: the tail split caches at most 63 positions
+        for (int m = warp; m < M; m += kAttnWarps) {
+            const float NEG = __int_as_float(0xFF800000);
+            const float v0 = lane < cnt ? sc[m * 68 + lane] : NEG;
+            const float v1 = lane + 32 < cnt ? sc[m * 68 + lane + 32] : NEG;
+            const float mx = warp_max(fmaxf(v0, v1));
+            const float p0 = lane < cnt ? exp2f(v0 - mx) : 0.f;
+            const float p1 = lane + 32 < cnt ? exp2f(v1 - mx) : 0.f;
+            if (lane < cnt) sc[m * 68 + lane] = p0;
+            if (lane + 32 < cnt) sc[m * 68 + lane + 32] = p1;
+            const float sum = warp_sum(p0 + p1);
+            if (lane == 0) { stat[2 * m] = mx; stat[2 * m + 1] = sum; }
+        }
+        __syncthreads();
+        if (tid < HD) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                float o = 0.f;
+                for (int t = 0; t < n_valid; ++t) o = fmaf(sc[m * 68 + t], bf16_bits_to_f32(vs[t * HD + tid]), o);
+                if (tail) o = fmaf(sc[m * 68 + n_valid], bf16_bits_to_f32(vtail[m * HD + tid]), o);
+                float* part = a.partial + (((size_t)m * H + h) * a.max_splits + s) * (HD + 2);
+                part[tid] = o;
+                if (tid == 0) { part[HD] = stat[2 * m]; part[HD + 1] = stat[2 * m + 1]; }
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- merge of the splits by the last CTA of this head
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) *flag = (atomicAdd(&a.tickets[h], 1) == G - 1);
+    __syncthreads();
+    if (!*flag) return;
+    __threadfence();
+    if (tid < HD) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float* part = a.partial + ((size_t)m * H + h) * a.max_splits * (HD + 2);
+            float mx = __int_as_float(0xFF800000);
+            for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldcg(part + (size_t)s * (HD + 2) + HD));
+            float num = 0.f, den = 0.f;
+            for (int s = 0; s < n_splits; ++s) {
+                const float* ps = part + (size_t)s * (HD + 2);
+                const float w = exp2f(__ldcg(ps + HD) - mx);
+                num = fmaf(__ldcg(ps + tid), w, num);
+                den = fmaf(__ldcg(ps + HD + 1), w, den);
+            }
+            a.out[(size_t)m * a.ldo + h * HD + tid] = num / den;
+        }
+    }
+    if (tid == 0) a.tickets[h] = 0;
+}
+
+size_t attn_partial_floats(int M, int H, int hd, int max_splits) {
+    return (size_t)M * H * max_splits * (hd + 2);
+}
+
+template <int M, int HD>
+static cudaError_t launch_attn(const AttnArgs& a, cudaStream_t st, bool pdl, int n_sms) {
+    using S = AttnSmem<HD>;
+    static bool configured = false;
+    auto kern = attn_kernel<M, HD>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    int G = (4 * n_sms + a.H - 1) / a.H;
+    if (G > a.max_splits) G = a.max_splits;
+    if (G < 1) G = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.H, G);
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = S::kBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <int HD>
+static cudaError_t launch_attn_m(const AttnArgs& a, cudaStream_t st, bool pdl, int n_sms) {
+    switch (a.M) {
+        case 1: return launch_attn<1, HD>(a, st, pdl, n_sms);
+        case 2: return launch_attn<2, HD>(a, st, pdl, n_sms);
+        case 3: return launch_attn<3, HD>(a, st, pdl, n_sms);
+        case 4: return launch_attn<4, HD>(a, st, pdl, n_sms);
+        case 5: return launch_attn<5, HD>(a, st, pdl, n_sms);
+        case 6: return launch_attn<6, HD>(a, st, pdl, n_sms);
+        case 7: return launch_attn<7, HD>(a, st, pdl, n_sms);
+        case 8: return launch_attn<8, HD>(a, st, pdl, n_sms);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st, bool pdl, int n_sms) {
+    if (a.hd == 128) return launch_attn_m<128>(a, st, pdl, n_sms);
+    if (a.hd == 64) return launch_attn_m<64>(a, st, pdl, n_sms);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace ppd

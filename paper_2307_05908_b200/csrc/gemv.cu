@@ -1,0 +1,369 @@
+// Skinny-M weight-streaming matrix product for decode: y[m][n] = sum_k W[n][k] x'[m][k], M <= 8.
+//
+// This one kernel shape covers the QKV, O, gate/up (SwiGLU), down and vocabulary-head products
+// of a decoder block applied to M token rows (M = 1 for the main pass, M = k for the candidate
+// branches of PPD, Algorithm 2).  It is bound by the HBM stream of the bf16 weights:
+//   * weights are pre-packed into 16 KB tiles (32 rows x 256 columns); a CTA owns whole row
+//     groups and a producer warp streams their tiles with bulk asynchronous copies (TMA) into a
+//     multi-stage shared-memory ring, together with the matching slice of the activations;
+//   * eight consumer warps each own four rows of the tile; a lane accumulates its eight columns
+//     of every chunk in a fixed order, so a row's result never depends on M or on other rows
+//     (batch invariance: PPD branches reproduce the main pass bit for bit);
+//   * RMSNorm of the input, the residual add, SwiGLU and the head's top-k are fused in;
+//   * the weight prefetch is issued before the programmatic-dependent-launch wait, so it
+//     overlaps the tail of the previous kernel.
+#include "common.cuh"
+#include "gemv.cuh"
+
+namespace ppd {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kRowsPerWarp = kTileRows / kConsumerWarps;  // 4
+constexpr int kGemvThreads = (kConsumerWarps + 1) * 32;
+constexpr int kTilesPerStage = 2;
+
+template <int M>
+struct GemvCfg {
+    static constexpr int kStages = (M == 1) ? 3 : 2;
+    static constexpr int kStageW = kTilesPerStage * kTileBytes;
+    static constexpr int kStageX = M * kTilesPerStage * kTileCols * 4;
+    static constexpr int kStageG = kTilesPerStage * kTileCols * 4;
+    static constexpr int kStageBytes = kStageW + kStageX + kStageG;
+    // ring | barriers (full, empty) | inv_rms[8] | warp partials [8][8] | head lists [8 warps][8 rows][8] (v,i)
+    static constexpr int kBarOff = kStages * kStageBytes;
+    static constexpr int kInvOff = kBarOff + 2 * kStages * 8;
+    static constexpr int kRedOff = kInvOff + kMaxRows * 4;
+    static constexpr int kListOff = kRedOff + kConsumerWarps * kMaxRows * 4;
+    static constexpr int kSmemBytes = kListOff + kConsumerWarps * kMaxRows * 8 * 8 + 16;
+};
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Inserts (nv, ni) into the descending list held by lanes 0..7 (lv, li).
+__device__ __forceinline__ void list_insert(float& lv, int& li, float nv, int ni, int lane) {
+    const unsigned ahead = __ballot_sync(0xFFFFFFFFu, lane < 8 && better(lv, li, nv, ni));
+    const int pos = __popc(ahead);
+    const float upv = __shfl_up_sync(0xFFFFFFFFu, lv, 1);
+    const int upi = __shfl_up_sync(0xFFFFFFFFu, li, 1);
+    if (lane < 8) {
+        if (lane > pos) { lv = upv; li = upi; }
+        else if (lane == pos) { lv = nv; li = ni; }
+    }
+}
+
+// Extracts the 8 best of `n` candidates (vals/ids in shared or global memory) in total order
+// into lanes 0..7 of the calling warp.  Ids are distinct.  Round r takes the best candidate
+// that is strictly worse than round r-1's winner, so nothing has to be marked.
+template <bool GLOBAL>
+__device__ __forceinline__ void select8(const float* vals, const int* ids, int n, int lane, float& ov, int& oi) {
+    float pv = __int_as_float(0x7F800000);  // +inf
+    int pi = -1;
+    ov = __int_as_float(0xFF800000);
+    oi = 0x7FFFFFFF;
+    for (int r = 0; r < 8; ++r) {
+        float bv = __int_as_float(0xFF800000);
+        int bi = 0x7FFFFFFF;
+        for (int c = lane; c < n; c += 32) {
+            const float v = GLOBAL ? __ldcg(vals + c) : vals[c];   // global lists were written by other CTAs
+            const int i = GLOBAL ? __ldcg(ids + c) : ids[c];
+            if (better(pv, pi, v, i) && better(v, i, bv, bi)) { bv = v; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v2 = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+            const int i2 = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+            if (better(v2, i2, bv, bi)) { bv = v2; bi = i2; }
+        }
+        if (lane == r) { ov = bv; oi = bi; }
+        pv = bv;
+        pi = bi;
+    }
+}
+
+template <int M, int MODE, bool NORM>
+__global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvArgs a) {
+    using C = GemvCfg<M>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
+    uint64_t* empty = full + C::kStages;
+    float* inv_rms = reinterpret_cast<float*>(smem + C::kInvOff);
+    float* red = reinterpret_cast<float*>(smem + C::kRedOff);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int n_rg = (a.N + kTileRows - 1) / kTileRows;
+    const int n_kc = (a.K + kTileCols - 1) / kTileCols;
+    const int spr = (n_kc + kTilesPerStage - 1) / kTilesPerStage;  // stages per row group
+    const int my_rgs = (n_rg > (int)blockIdx.x) ? (n_rg - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total = my_rgs * spr;
+
+    if (tid == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kConsumerWarps);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            auto stage_geom = [&](int it, int& rg, int& c0, int& nt) {
+                rg = (int)blockIdx.x + (it / spr) * (int)gridDim.x;
+                c0 = (it % spr) * kTilesPerStage;
+                nt = min(kTilesPerStage, n_kc - c0);
+            };
+            auto issue_w = [&](int it) {
+                int rg, c0, nt;
+                stage_geom(it, rg, c0, nt);
+                const int slot = it % C::kStages;
+                uint8_t* st = smem + slot * C::kStageBytes;
+                const uint32_t bytes = nt * kTileBytes + M * nt * kTileCols * 4 + (NORM ? nt * kTileCols * 4 : 0);
+                mbar_arrive_expect_tx(&full[slot], bytes);
+                bulk_g2s(st, a.w + ((size_t)rg * n_kc + c0) * kTileElems, nt * kTileBytes, &full[slot]);
+            };
+            auto issue_x = [&](int it) {
+                int rg, c0, nt;
+                stage_geom(it, rg, c0, nt);
+                const int slot = it % C::kStages;
+                uint8_t* st = smem + slot * C::kStageBytes;
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+                    bulk_g2s(st + C::kStageW + m * kTilesPerStage * kTileCols * 4,
+                             a.x + (size_t)m * a.ldx + (size_t)c0 * kTileCols, nt * kTileCols * 4, &full[slot]);
+                if (NORM)
+                    bulk_g2s(st + C::kStageW + C::kStageX, a.gain + (size_t)c0 * kTileCols, nt * kTileCols * 4,
+                             &full[slot]);
+            };
+            const int pre = min(C::kStages, total);
+            for (int it = 0; it < pre; ++it) issue_w(it);   // weights do not depend on the previous kernel
+            pdl_wait();
+            for (int it = 0; it < pre; ++it) issue_x(it);
+            for (int it = pre; it < total; ++it) {
+                const int slot = it % C::kStages;
+                mbar_wait(&empty[slot], ((it / C::kStages) - 1) & 1, a.err, kErrEmptyWait);
+                issue_w(it);
+                issue_x(it);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    pdl_wait();
+    if (NORM) {
+        // 1/rms of each input row; fixed reduction order (thread-strided, warp tree, 8 warps in order)
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float* xr = a.x + (size_t)m * a.ldx;
+            float ss = 0.f;
+            for (int i = tid; i < a.K; i += kConsumerWarps * 32) ss = fmaf(xr[i], xr[i], ss);
+            ss = warp_sum(ss);
+            if (lane == 0) red[warp * kMaxRows + m] = ss;
+        }
+        consumer_sync();
+        if (tid < M) {
+            float ss = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) ss += red[w * kMaxRows + tid];
+            inv_rms[tid] = 1.0f / sqrtf(ss / (float)a.K + a.eps);
+        }
+        consumer_sync();
+    }
+    float inv[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) inv[m] = NORM ? inv_rms[m] : 1.f;
+
+    // head: running top-8 of this warp, one list per row, held by lanes 0..7
+    float lv[M];
+    int li[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) { lv[m] = __int_as_float(0xFF800000); li[m] = 0x7FFFFFFF; }
+
+    const int r0 = warp * kRowsPerWarp;
+    int it = 0;
+    for (int rg = blockIdx.x; rg < n_rg; rg += gridDim.x) {
+        float acc[M][kRowsPerWarp];
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+            for (int r = 0; r < kRowsPerWarp; ++r) acc[m][r] = 0.f;
+
+        for (int c0 = 0; c0 < n_kc; c0 += kTilesPerStage, ++it) {
+            const int slot = it % C::kStages;
+            mbar_wait(&full[slot], (it / C::kStages) & 1, a.err, kErrFullWait);
+            const uint8_t* st = smem + slot * C::kStageBytes;
+            const int nt = min(kTilesPerStage, n_kc - c0);
+            for (int t = 0; t < nt; ++t) {
+                float xv[M][8];
+                float gs[8];
+                if (NORM) {
+                    const float4* gp = reinterpret_cast<const float4*>(st + C::kStageW + C::kStageX) + t * (kTileCols / 4) + lane * 2;
+                    const float4 g0 = gp[0], g1 = gp[1];
+                    gs[0] = g0.x; gs[1] = g0.y; gs[2] = g0.z; gs[3] = g0.w;
+                    gs[4] = g1.x; gs[5] = g1.y; gs[6] = g1.z; gs[7] = g1.w;
+                }
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    const float4* xp = reinterpret_cast<const float4*>(st + C::kStageW) +
+                                       (m * kTilesPerStage + t) * (kTileCols / 4) + lane * 2;
+                    const float4 x0 = xp[0], x1 = xp[1];
+                    xv[m][0] = x0.x; xv[m][1] = x0.y; xv[m][2] = x0.z; xv[m][3] = x0.w;
+                    xv[m][4] = x1.x; xv[m][5] = x1.y; xv[m][6] = x1.z; xv[m][7] = x1.w;
+                    if (NORM) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) xv[m][j] = __fmul_rn(xv[m][j], __fmul_rn(gs[j], inv[m]));
+                    }
+                }
+                const uint4* wt = reinterpret_cast<const uint4*>(st + t * kTileBytes) + r0 * 32 + lane;
+#pragma unroll
+                for (int r = 0; r < kRowsPerWarp; ++r) {
+                    const uint4 w = wt[r * 32];
+                    float wf[8];
+                    wf[0] = bf16_lo(w.x); wf[1] = bf16_hi(w.x); wf[2] = bf16_lo(w.y); wf[3] = bf16_hi(w.y);
+                    wf[4] = bf16_lo(w.z); wf[5] = bf16_hi(w.z); wf[6] = bf16_lo(w.w); wf[7] = bf16_hi(w.w);
+#pragma unroll
+                    for (int m = 0; m < M; ++m)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[m][r] = fmaf(wf[j], xv[m][j], acc[m][r]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[slot]);
+        }
+
+        // ---- row-group epilogue
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+            for (int r = 0; r < kRowsPerWarp; ++r) acc[m][r] = warp_sum(acc[m][r]);
+        const int n0 = rg * kTileRows + r0;
+        if (MODE == kStore || MODE == kResid || MODE == kHead) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const float v = lane == 0 ? acc[m][0] : lane == 1 ? acc[m][1] : lane == 2 ? acc[m][2] : acc[m][3];
+                const int n = n0 + lane;
+                if (lane < kRowsPerWarp && n < a.N) {
+                    const size_t o = (size_t)m * a.ldo + n;
+                    a.out[o] = (MODE == kResid) ? a.resid[o] + v : v;
+                }
+                if (MODE == kHead) {
+#pragma unroll
+                    for (int r = 0; r < kRowsPerWarp; ++r)
+                        if (n0 + r < a.N) list_insert(lv[m], li[m], acc[m][r], n0 + r, lane);
+                }
+            }
+        } else {  // kSwiglu: rows (2j, 2j+1) = (gate_j, up_j)
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const float g = lane == 0 ? acc[m][0] : acc[m][2];
+                const float u = lane == 0 ? acc[m][1] : acc[m][3];
+                const int j = (n0 >> 1) + lane;
+                if (lane < 2 && 2 * j + 1 < a.N) a.out[(size_t)m * a.ldo + j] = (g / (1.0f + expf(-g))) * u;
+            }
+        }
+    }
+
+    if (MODE == kHead) {
+        // CTA merge of the 8 warp lists, then grid merge by the last CTA to arrive (no spinning).
+        float* cv = reinterpret_cast<float*>(smem + C::kListOff);                       // [8 warps][8 rows][8]
+        int* ci = reinterpret_cast<int*>(smem + C::kListOff + kConsumerWarps * kMaxRows * 8 * 4);
+        int* flag = reinterpret_cast<int*>(smem + C::kListOff + kConsumerWarps * kMaxRows * 8 * 8);
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+            if (lane < 8) {
+                cv[(m * kConsumerWarps + warp) * 8 + lane] = lv[m];
+                ci[(m * kConsumerWarps + warp) * 8 + lane] = li[m];
+            }
+        consumer_sync();
+        int* ticket = reinterpret_cast<int*>(a.head_scratch);
+        float* gv = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.head_scratch) + 256);  // [8 rows][ctas][8]
+        int* gi = reinterpret_cast<int*>(gv + (size_t)kMaxRows * kHeadMaxCtas * 8);
+        if (warp < M) {
+            float ov; int oi;
+            select8<false>(cv + warp * kConsumerWarps * 8, ci + warp * kConsumerWarps * 8, kConsumerWarps * 8, lane, ov, oi);
+            if (lane < 8) {
+                gv[((size_t)warp * kHeadMaxCtas + blockIdx.x) * 8 + lane] = ov;
+                gi[((size_t)warp * kHeadMaxCtas + blockIdx.x) * 8 + lane] = oi;
+            }
+        }
+        __threadfence();
+        consumer_sync();
+        if (tid == 0) {
+            const int t = atomicAdd(ticket, 1);
+            *flag = (t == (int)gridDim.x - 1);
+        }
+        consumer_sync();
+        if (*flag) {
+            __threadfence();
+            if (warp < M) {
+                float ov; int oi;
+                // the lists of row `warp` are contiguous: [ctas][8]
+                select8<true>(gv + (size_t)warp * kHeadMaxCtas * 8, gi + (size_t)warp * kHeadMaxCtas * 8, (int)gridDim.x * 8,
+                        lane, ov, oi);
+                if (lane < 8) {
+                    a.top_vals[warp * 8 + lane] = ov;
+                    a.top_ids[warp * 8 + lane] = oi;
+                }
+            }
+            if (tid == 0) *ticket = 0;  // ready for the next launch
+        }
+    }
+}
+
+template <int M, int MODE, bool NORM>
+static cudaError_t launch_one(const GemvArgs& a, cudaStream_t st, bool pdl, int n_sms) {
+    using C = GemvCfg<M>;
+    static bool configured = false;
+    auto kern = gemv_kernel<M, MODE, NORM>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int n_rg = (a.N + kTileRows - 1) / kTileRows;
+    int grid = n_rg < n_sms ? n_rg : n_sms;
+    if (MODE == kHead && grid > kHeadMaxCtas) grid = kHeadMaxCtas;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <int M>
+static cudaError_t launch_m(const GemvArgs& a, int mode, cudaStream_t st, bool pdl, int n_sms) {
+    const bool norm = a.gain != nullptr;
+    switch (mode) {
+        case kStore: return norm ? launch_one<M, kStore, true>(a, st, pdl, n_sms) : launch_one<M, kStore, false>(a, st, pdl, n_sms);
+        case kResid: return norm ? launch_one<M, kResid, true>(a, st, pdl, n_sms) : launch_one<M, kResid, false>(a, st, pdl, n_sms);
+        case kSwiglu: return norm ? launch_one<M, kSwiglu, true>(a, st, pdl, n_sms) : launch_one<M, kSwiglu, false>(a, st, pdl, n_sms);
+        case kHead: return norm ? launch_one<M, kHead, true>(a, st, pdl, n_sms) : launch_one<M, kHead, false>(a, st, pdl, n_sms);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_gemv(const GemvArgs& a, int M, int mode, cudaStream_t st, bool pdl, int n_sms) {
+    switch (M) {
+        case 1: return launch_m<1>(a, mode, st, pdl, n_sms);
+        case 2: return launch_m<2>(a, mode, st, pdl, n_sms);
+        case 3: return launch_m<3>(a, mode, st, pdl, n_sms);
+        case 4: return launch_m<4>(a, mode, st, pdl, n_sms);
+        case 5: return launch_m<5>(a, mode, st, pdl, n_sms);
+        case 6: return launch_m<6>(a, mode, st, pdl, n_sms);
+        case 7: return launch_m<7>(a, mode, st, pdl, n_sms);
+        case 8: return launch_m<8>(a, mode, st, pdl, n_sms);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace ppd

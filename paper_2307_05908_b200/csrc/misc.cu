@@ -1,0 +1,179 @@
+// Small kernels around the weight-streaming path: embedding gather, weight packing, RoPE table,
+// and PPD's verify/commit step.
+#include "common.cuh"
+#include "misc.cuh"
+
+namespace ppd {
+
+// ---------------------------------------------------------------- embedding gather  h_0 = E[x]
+__global__ void embed_kernel(const uint16_t* __restrict__ E, const int* __restrict__ tokens, int D, float* h, int ldh) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const uint16_t* e = E + (size_t)tokens[m] * D;
+    for (int i = threadIdx.x; i < D; i += blockDim.x) h[(size_t)m * ldh + i] = bf16_bits_to_f32(e[i]);
+}
+
+cudaError_t launch_embed(const uint16_t* E, const int* tokens, int M, int D, float* h, int ldh, cudaStream_t st, bool pdl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(M);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, embed_kernel, E, tokens, D, h, ldh);
+}
+
+// ---------------------------------------------------------------- weight packing
+// Source element (r, c) of a row-major matrix goes to packed row r*row_mul + row_off, i.e. tile
+// (row/32, c/256), position (row%32, c%256).  SRC_F32: the source is float32 and is rounded to bf16.
+template <bool SRC_F32>
+__global__ void pack_kernel(const void* __restrict__ src, int n_rows, int n_cols, uint16_t* __restrict__ dst,
+                            int row_mul, int row_off) {
+    const int n_kc = (n_cols + kTileCols - 1) / kTileCols;
+    const size_t total = (size_t)n_rows * n_cols;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / n_cols), c = (int)(i % n_cols);
+        const int pr = r * row_mul + row_off;
+        const uint16_t v = SRC_F32 ? f32_to_bf16_bits(reinterpret_cast<const float*>(src)[i])
+                                   : reinterpret_cast<const uint16_t*>(src)[i];
+        dst[((size_t)(pr / kTileRows) * n_kc + c / kTileCols) * kTileElems + (pr % kTileRows) * kTileCols + (c % kTileCols)] = v;
+    }
+}
+
+cudaError_t launch_pack(const void* src, bool src_f32, int n_rows, int n_cols, uint16_t* dst, int row_mul, int row_off,
+                        cudaStream_t st) {
+    const size_t total = (size_t)n_rows * n_cols;
+    int grid = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+    if (grid < 1) grid = 1;
+    if (src_f32) pack_kernel<true><<<grid, 256, 0, st>>>(src, n_rows, n_cols, dst, row_mul, row_off);
+    else pack_kernel<false><<<grid, 256, 0, st>>>(src, n_rows, n_cols, dst, row_mul, row_off);
+    return cudaGetLastError();
+}
+
+// plain conversion to float32 (norm gains) or to bf16 bits (embedding table)
+template <bool SRC_F32, bool DST_F32>
+__global__ void convert_kernel(const void* __restrict__ src, void* __restrict__ dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        if (DST_F32) {
+            reinterpret_cast<float*>(dst)[i] = SRC_F32 ? reinterpret_cast<const float*>(src)[i]
+                                                       : bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(src)[i]);
+        } else {
+            reinterpret_cast<uint16_t*>(dst)[i] = SRC_F32 ? f32_to_bf16_bits(reinterpret_cast<const float*>(src)[i])
+                                                          : reinterpret_cast<const uint16_t*>(src)[i];
+        }
+    }
+}
+
+cudaError_t launch_convert(const void* src, bool src_f32, void* dst, bool dst_f32, size_t n, cudaStream_t st) {
+    int grid = (int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096);
+    if (grid < 1) grid = 1;
+    if (src_f32 && dst_f32) convert_kernel<true, true><<<grid, 256, 0, st>>>(src, dst, n);
+    else if (src_f32) convert_kernel<true, false><<<grid, 256, 0, st>>>(src, dst, n);
+    else if (dst_f32) convert_kernel<false, true><<<grid, 256, 0, st>>>(src, dst, n);
+    else convert_kernel<false, false><<<grid, 256, 0, st>>>(src, dst, n);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- RoPE table
+// table[pos][i] = (cos, sin)(pos * theta^(-2i/hd)), evaluated in double so that large positions
+// keep full float accuracy.
+__global__ void rope_table_kernel(float2* table, int n_pos, int hd, double theta) {
+    const int half = hd / 2;
+    const size_t total = (size_t)n_pos * half;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int pos = (int)(i / half), j = (int)(i % half);
+        const double ang = (double)pos * pow(theta, -2.0 * (double)j / (double)hd);
+        table[i] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+}
+
+cudaError_t launch_rope_table(float2* table, int n_pos, int hd, double theta, cudaStream_t st) {
+    rope_table_kernel<<<256, 256, 0, st>>>(table, n_pos, hd, theta);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- verify / commit (Algorithm 2)
+// Compares the final argmax with the k early candidates.  On a match with candidate i* the
+// branch's hidden state after b layers becomes the main hidden state and its K/V of layers
+// 1..b move from branch slot i* into the cache at position pos+1; otherwise everything
+// speculative is dropped.  Then the token is emitted and the position advances.  Every CTA
+// recomputes the decision; CTA c copies layers c, c+grid, ...; the last CTA to finish (atomic
+// ticket, no spinning) advances the state, so no CTA can observe the new position early.
+__global__ void commit_kernel(const CommitArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ int s_last;
+    const int token = a.final_ids[0];
+    int istar = -1;
+    for (int i = 0; i < a.k; ++i)
+        if (a.cand[i] == token) istar = i;
+    const int pos = *a.d_pos;
+    if (istar >= 0) {
+        const int np = pos + 1;
+        const int page = a.page_table[np / kPageTokens];
+        const int hw = a.hd / 2;  // 32-bit words per head row
+        const size_t page_elems = (size_t)2 * a.H * kPageTokens * a.hd;
+        for (int l = blockIdx.x; l < a.b; l += gridDim.x) {
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(a.slots + (size_t)istar * a.slot_stride + (size_t)l * a.slot_layer_stride);
+            uint16_t* pg = a.kv + (size_t)l * a.kv_layer_stride + (size_t)page * page_elems;
+            // words: [kv][h][hd/2]
+            for (int w = threadIdx.x; w < 2 * a.H * hw; w += blockDim.x) {
+                const int kv = w / (a.H * hw), rem = w % (a.H * hw), h = rem / hw, j = rem % hw;
+                uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)(kv * a.H + h) * kPageTokens + (np % kPageTokens)) * a.hd);
+                dst[j] = src[w];
+            }
+        }
+        if (blockIdx.x == 0)
+            for (int i = threadIdx.x; i < a.D; i += blockDim.x) a.h_main[i] = a.h_branch[(size_t)istar * a.ldh + i];
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(a.ticket, 1) == (int)gridDim.x - 1);
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {
+        const int step = *a.d_step;
+        a.out_tokens[step] = token;
+        a.out_hit[step] = istar >= 0 ? 1 : 0;
+        a.out_margin[step] = a.final_vals[0] - a.final_vals[1];
+        a.last[0] = token;
+        a.last[1] = istar >= 0 ? 1 : 0;
+        *a.d_pending = token;
+        *a.d_pos = pos + 1;
+        *a.d_step = step + 1;
+        *a.ticket = 0;
+    }
+}
+
+cudaError_t launch_commit(const CommitArgs& a, cudaStream_t st, bool pdl) {
+    int grid = a.k > 0 && a.b > 0 ? (a.b < 16 ? a.b : 16) : 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, commit_kernel, a);
+}
+
+// sets the small device state block
+__global__ void set_state_kernel(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step) {
+    if (threadIdx.x == 0) {
+        if (d_pos) *d_pos = pos;
+        if (d_pending) *d_pending = pending;
+        if (d_step) *d_step = step;
+    }
+}
+
+cudaError_t launch_set_state(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step, cudaStream_t st) {
+    set_state_kernel<<<1, 32, 0, st>>>(d_pos, pos, d_pending, pending, d_step, step);
+    return cudaGetLastError();
+}
+
+}  // namespace ppd

@@ -1,0 +1,42 @@
+// Launchers of the small kernels (internal to the library).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ppd {
+
+struct CommitArgs {
+    const int* final_ids;     // [8] top ids of the final head (argmax first)
+    const float* final_vals;  // [8]
+    const int* cand;          // [8] early candidates
+    int k;                    // number of candidates (0 = plain greedy step)
+    int b;                    // branch depth in layers
+    int H, hd, D;
+    const uint16_t* slots;    // branch slots: slot i, layer l at slots + i*slot_stride + l*slot_layer_stride, [2][H][hd]
+    long long slot_stride, slot_layer_stride;
+    uint16_t* kv;             // cache: layer l at kv + l*kv_layer_stride; page = [2][H][64][hd]
+    long long kv_layer_stride;
+    const int* page_table;
+    const float* h_branch;    // [k][ldh] hidden states of the branches after b layers
+    int ldh;
+    float* h_main;            // [D] receives the committed hidden state
+    int* d_pos;
+    int* d_pending;
+    int* d_step;
+    int* ticket;
+    int* out_tokens;          // [max_steps]
+    uint8_t* out_hit;         // [max_steps]
+    float* out_margin;        // [max_steps] top-1 minus top-2 final logit
+    int* last;                // [2] (token, hit) of this step
+};
+
+cudaError_t launch_embed(const uint16_t* E, const int* tokens, int M, int D, float* h, int ldh, cudaStream_t st, bool pdl);
+cudaError_t launch_pack(const void* src, bool src_f32, int n_rows, int n_cols, uint16_t* dst, int row_mul, int row_off,
+                        cudaStream_t st);
+cudaError_t launch_convert(const void* src, bool src_f32, void* dst, bool dst_f32, size_t n, cudaStream_t st);
+cudaError_t launch_rope_table(float2* table, int n_pos, int hd, double theta, cudaStream_t st);
+cudaError_t launch_commit(const CommitArgs& a, cudaStream_t st, bool pdl);
+cudaError_t launch_set_state(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step, cudaStream_t st);
+
+}  // namespace ppd

@@ -1,0 +1,702 @@
+// C ABI of the library: context inside a caller-owned device arena, weight upload and packing,
+// prefill, greedy step, and the PPD step scheduler (Algorithm 2 on two CUDA streams: the main
+// pass and the k candidate branches overlap between the early head and the verify/commit kernel).
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/ppd.h"
+#include "common.cuh"
+#include "gemv.cuh"
+#include "misc.cuh"
+
+using namespace ppd;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kStagingBytes = 64ull << 20;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    int Dp, Fp, n_pages, max_splits;
+    // per-layer weight block (byte offsets inside the block)
+    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, layer_bytes;
+    size_t emb, layers, g_final, w_head, weights_end;
+    size_t rope, kv, page_table, slots;
+    long long kv_layer_elems, slot_elems, slot_layer_elems;
+    size_t ws[2];            // main / branch workspaces
+    size_t ws_h, ws_qkv, ws_attn, ws_z, ws_part, ws_tick, ws_bytes[2];   // offsets inside a workspace
+    size_t logits_final, logits_early, top_final, top_early, head_scratch;
+    size_t state, prompt, out_tokens, out_hit, out_margin, staging, total;
+};
+
+bool valid_config(const ppd_config* c) {
+    if (!c) return false;
+    if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ffn < 8 || c->vocab < 8) return false;
+    if (c->n_heads * c->head_dim != c->d_model) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->d_model % 8 || c->d_ffn % 8) return false;   // 16-byte rows
+    if (c->max_seq < 2 || c->max_k < 0 || c->max_k > PPD_MAX_K) return false;
+    if (c->kv_page_tokens != kPageTokens) return false;
+    if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+    return true;
+}
+
+Layout plan(const ppd_config& c) {
+    Layout L{};
+    const size_t D = c.d_model, F = c.d_ffn, V = c.vocab;
+    L.Dp = round_up(c.d_model, kTileCols);
+    L.Fp = round_up(c.d_ffn, kTileCols);
+    L.n_pages = (c.max_seq + kPageTokens - 1) / kPageTokens;
+    L.max_splits = L.n_pages;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, kAlign); return r; };
+    // layer block
+    {
+        size_t lo = 0;
+        auto ltake = [&](size_t bytes) { size_t r = lo; lo = align_up(lo + bytes, kAlign); return r; };
+        L.off_wqkv = ltake(ppd_packed_bytes(3 * (int)D, (int)D));
+        L.off_wo = ltake(ppd_packed_bytes((int)D, (int)D));
+        L.off_wgu = ltake(ppd_packed_bytes(2 * (int)F, (int)D));
+        L.off_wd = ltake(ppd_packed_bytes((int)D, (int)F));
+        L.off_g1 = ltake((size_t)L.Dp * 4);
+        L.off_g2 = ltake((size_t)L.Dp * 4);
+        L.layer_bytes = lo;
+    }
+    L.emb = take(V * D * 2);
+    L.layers = take(L.layer_bytes * c.n_layers);
+    L.g_final = take((size_t)L.Dp * 4);
+    L.w_head = take(ppd_packed_bytes((int)V, (int)D));
+    L.weights_end = o;
+    L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
+    L.kv_layer_elems = (long long)L.n_pages * 2 * c.n_heads * kPageTokens * c.head_dim;
+    L.kv = take((size_t)c.n_layers * L.kv_layer_elems * 2);
+    L.page_table = take((size_t)L.n_pages * 4);
+    L.slot_layer_elems = 2ll * c.n_heads * c.head_dim;
+    L.slot_elems = L.slot_layer_elems * c.n_layers;
+    L.slots = take((size_t)(c.max_k > 0 ? c.max_k : 1) * L.slot_elems * 2);
+    for (int w = 0; w < 2; ++w) {
+        const size_t rows = c.max_k > 0 ? c.max_k : 1;   // same offsets in both workspaces
+        size_t wo = 0;
+        auto wtake = [&](size_t bytes) { size_t r = wo; wo = align_up(wo + bytes, kAlign); return r; };
+        L.ws_h = wtake(kMaxRows * (size_t)L.Dp * 4);
+        L.ws_qkv = wtake(kMaxRows * 3 * D * 4);
+        L.ws_attn = wtake(kMaxRows * (size_t)L.Dp * 4);
+        L.ws_z = wtake(kMaxRows * (size_t)L.Fp * 4);
+        L.ws_part = wo;
+        wo = align_up(wo + attn_partial_floats((int)rows, c.n_heads, c.head_dim, L.max_splits) * 4, kAlign);
+        L.ws_tick = wo;
+        wo = align_up(wo + (size_t)c.n_heads * 4, kAlign);
+        L.ws_bytes[w] = wo;
+        L.ws[w] = take(wo);
+    }
+    L.logits_final = take(V * 4);
+    L.logits_early = take(V * 4);
+    L.top_final = take(64 * 4);      // ids[8] at +0, vals[8] at +128 bytes
+    L.top_early = take(64 * 4);
+    L.head_scratch = take(kHeadScratchBytes);
+    L.state = take(256);
+    L.prompt = take((size_t)c.max_seq * 4);
+    L.out_tokens = take((size_t)c.max_seq * 4);
+    L.out_hit = take((size_t)c.max_seq);
+    L.out_margin = take((size_t)c.max_seq * 4);
+    L.staging = take(kStagingBytes);
+    L.total = o;
+    return L;
+}
+
+// indices into the device state block (ints)
+enum { S_POS = 0, S_PENDING = 1, S_STEP = 2, S_TICKET = 3, S_LAST_TOKEN = 4, S_LAST_HIT = 5, S_ERR = 6 };
+
+struct Lane {      // one activation workspace (main: 1 row, branch: up to max_k rows)
+    float *h, *qkv, *attn, *z, *partial;
+    int* tickets;
+};
+
+}  // namespace
+
+struct ppd_ctx {
+    ppd_config c;
+    Layout L;
+    uint8_t* base;
+    cudaStream_t sm, sb;
+    cudaEvent_t ev_early, ev_branch, ev_t0, ev_t1;
+    int n_sms;
+    bool loaded, prefilled, pdl;
+    int pos, pending;     // host mirrors
+    bool prev_hit;
+    int prev_b;           // branch depth of the step that produced prev_hit
+    int* h_last;          // pinned host: (token, hit, err)
+    ppd_stats stats;
+    cudaError_t cuda_err;
+    Lane lane[2];
+    int* state;
+};
+
+namespace {
+
+template <typename T>
+T* at(ppd_ctx* x, size_t off) { return reinterpret_cast<T*>(x->base + off); }
+
+int fail_cuda(ppd_ctx* x, cudaError_t e) {
+    if (x) x->cuda_err = e;
+    return PPD_ECUDA;
+}
+
+#define CK(expr)                                       \
+    do {                                               \
+        cudaError_t e__ = (expr);                      \
+        if (e__ != cudaSuccess) return fail_cuda(x, e__); \
+    } while (0)
+
+uint8_t* layer_block(ppd_ctx* x, int l) { return x->base + x->L.layers + (size_t)l * x->L.layer_bytes; }
+
+// Decoder blocks [l0, l1) applied to M rows of a lane.  The rows sit at position
+// (d_pos ? *d_pos : 0) + pos_off; branch rows keep their K/V in their slots.
+int run_layers(ppd_ctx* x, int lane_id, int M, int l0, int l1, const int* d_pos, int pos_off, bool branch, cudaStream_t st) {
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    Lane& ln = x->lane[lane_id];
+    const int D = c.d_model, F = c.d_ffn;
+    int* err = x->state + S_ERR;
+    for (int l = l0; l < l1; ++l) {
+        uint8_t* lb = layer_block(x, l);
+        GemvArgs g{};
+        g.err = err;
+        g.eps = c.rms_eps;
+        // q|k|v = Wqkv . RMSNorm(h)
+        g.w = reinterpret_cast<const uint16_t*>(lb + L.off_wqkv); g.N = 3 * D; g.K = D;
+        g.x = ln.h; g.ldx = L.Dp; g.gain = reinterpret_cast<const float*>(lb + L.off_g1);
+        g.out = ln.qkv; g.ldo = 3 * D; g.resid = nullptr;
+        CK(launch_gemv(g, M, kStore, st, x->pdl, x->n_sms));
+        AttnArgs a{};
+        a.qkv = ln.qkv; a.M = M; a.H = c.n_heads; a.hd = c.head_dim; a.d_pos = d_pos; a.pos_off = pos_off;
+        a.kv_layer = at<uint16_t>(x, L.kv) + (size_t)l * L.kv_layer_elems;
+        a.page_table = at<int>(x, L.page_table);
+        a.slots = branch ? at<uint16_t>(x, L.slots) + (size_t)l * L.slot_layer_elems : nullptr;
+        a.slot_stride = L.slot_elems;
+        a.rope = at<float2>(x, L.rope);
+        a.partial = ln.partial; a.max_splits = L.max_splits; a.tickets = ln.tickets;
+        a.out = ln.attn; a.ldo = L.Dp; a.err = err;
+        CK(launch_attention(a, st, x->pdl, x->n_sms));
+        // h += Wo . attn
+        g.w = reinterpret_cast<const uint16_t*>(lb + L.off_wo); g.N = D; g.K = D;
+        g.x = ln.attn; g.ldx = L.Dp; g.gain = nullptr; g.resid = ln.h; g.out = ln.h; g.ldo = L.Dp;
+        CK(launch_gemv(g, M, kResid, st, x->pdl, x->n_sms));
+        // z = silu(Wg n) * (Wu n), n = RMSNorm(h)
+        g.w = reinterpret_cast<const uint16_t*>(lb + L.off_wgu); g.N = 2 * F; g.K = D;
+        g.x = ln.h; g.ldx = L.Dp; g.gain = reinterpret_cast<const float*>(lb + L.off_g2); g.resid = nullptr;
+        g.out = ln.z; g.ldo = L.Fp;
+        CK(launch_gemv(g, M, kSwiglu, st, x->pdl, x->n_sms));
+        // h += Wd . z
+        g.w = reinterpret_cast<const uint16_t*>(lb + L.off_wd); g.N = D; g.K = F;
+        g.x = ln.z; g.ldx = L.Fp; g.gain = nullptr; g.resid = ln.h; g.out = ln.h; g.ldo = L.Dp;
+        CK(launch_gemv(g, M, kResid, st, x->pdl, x->n_sms));
+        x->stats.kernel_launches += 5;
+    }
+    return PPD_OK;
+}
+
+// logits = W_H . RMSNorm_final(h of the main lane); top-8 into `top` (ids at +0, values at +32 ints)
+int run_head(ppd_ctx* x, size_t logits_off, size_t top_off, cudaStream_t st) {
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    GemvArgs g{};
+    g.err = x->state + S_ERR;
+    g.eps = c.rms_eps;
+    g.w = at<uint16_t>(x, L.w_head); g.N = c.vocab; g.K = c.d_model;
+    g.x = x->lane[0].h; g.ldx = L.Dp; g.gain = at<float>(x, L.g_final);
+    g.out = at<float>(x, logits_off); g.ldo = c.vocab;
+    g.head_scratch = at<void>(x, L.head_scratch);
+    g.top_ids = at<int>(x, top_off);
+    g.top_vals = at<float>(x, top_off) + 32;
+    CK(launch_gemv(g, 1, kHead, st, x->pdl, x->n_sms));
+    x->stats.kernel_launches += 1;
+    return PPD_OK;
+}
+
+int run_commit(ppd_ctx* x, int k, int b, cudaStream_t st) {
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    CommitArgs a{};
+    a.final_ids = at<int>(x, L.top_final);
+    a.final_vals = at<float>(x, L.top_final) + 32;
+    a.cand = at<int>(x, L.top_early);
+    a.k = k; a.b = b; a.H = c.n_heads; a.hd = c.head_dim; a.D = c.d_model;
+    a.slots = at<uint16_t>(x, L.slots); a.slot_stride = L.slot_elems; a.slot_layer_stride = L.slot_layer_elems;
+    a.kv = at<uint16_t>(x, L.kv); a.kv_layer_stride = L.kv_layer_elems;
+    a.page_table = at<int>(x, L.page_table);
+    a.h_branch = x->lane[1].h; a.ldh = L.Dp; a.h_main = x->lane[0].h;
+    a.d_pos = x->state + S_POS; a.d_pending = x->state + S_PENDING; a.d_step = x->state + S_STEP;
+    a.ticket = x->state + S_TICKET;
+    a.out_tokens = at<int>(x, L.out_tokens); a.out_hit = at<uint8_t>(x, L.out_hit); a.out_margin = at<float>(x, L.out_margin);
+    a.last = x->state + S_LAST_TOKEN;
+    CK(launch_commit(a, st, x->pdl));
+    x->stats.kernel_launches += 1;
+    return PPD_OK;
+}
+
+// Reads (token, hit, err) of the step just enqueued; synchronises the main stream.
+int finish_step(ppd_ctx* x, int32_t* token, uint8_t* hit) {
+    CK(cudaMemcpyAsync(x->h_last, x->state + S_LAST_TOKEN, 3 * sizeof(int), cudaMemcpyDeviceToHost, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    if (x->h_last[2] != 0) return PPD_ETIMEOUT;
+    *token = x->h_last[0];
+    *hit = (uint8_t)x->h_last[1];
+    return PPD_OK;
+}
+
+// One decode step.  k = 0: conventional greedy step.  k >= 1: PPD step with early layer l.
+int decode_step(ppd_ctx* x, int k, int l, int32_t* token, uint8_t* hit) {
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    const int d = c.n_layers;
+    int* d_pos = x->state + S_POS;
+    CK(cudaEventRecord(x->ev_t0, x->sm));
+    // After a hit, layers 1..prev_b of the pending token were committed from its branch.  If this
+    // step's early layer lies below that depth (l changed between calls) the token is recomputed
+    // from layer 1, which rewrites the same values.
+    const bool cont = x->prev_hit && !(k > 0 && x->prev_b > l);
+    const int start = cont ? x->prev_b : 0;
+    int rc;
+    if (!cont) {
+        CK(launch_embed(at<uint16_t>(x, L.emb), x->state + S_PENDING, 1, c.d_model, x->lane[0].h, L.Dp, x->sm, x->pdl));
+        x->stats.kernel_launches += 1;
+    }
+    int b = 0;
+    if (k == 0) {
+        if ((rc = run_layers(x, 0, 1, start, d, d_pos, 0, false, x->sm))) return rc;
+    } else {
+        b = l < d - l ? l : d - l;
+        if ((rc = run_layers(x, 0, 1, start, l, d_pos, 0, false, x->sm))) return rc;
+        if ((rc = run_head(x, L.logits_early, L.top_early, x->sm))) return rc;
+        CK(cudaEventRecord(x->ev_early, x->sm));
+        // candidate branches: k rows through layers 1..b at position pos+1
+        CK(cudaStreamWaitEvent(x->sb, x->ev_early, 0));
+        CK(launch_embed(at<uint16_t>(x, L.emb), at<int>(x, L.top_early), k, c.d_model, x->lane[1].h, L.Dp, x->sb, false));
+        x->stats.kernel_launches += 1;
+        if ((rc = run_layers(x, 1, k, 0, b, d_pos, 1, true, x->sb))) return rc;
+        CK(cudaEventRecord(x->ev_branch, x->sb));
+        // main tail
+        if ((rc = run_layers(x, 0, 1, l, d, d_pos, 0, false, x->sm))) return rc;
+    }
+    if ((rc = run_head(x, L.logits_final, L.top_final, x->sm))) return rc;
+    if (k > 0) CK(cudaStreamWaitEvent(x->sm, x->ev_branch, 0));
+    if ((rc = run_commit(x, k, b, x->sm))) return rc;
+    CK(cudaEventRecord(x->ev_t1, x->sm));
+    if ((rc = finish_step(x, token, hit))) return rc;
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, x->ev_t0, x->ev_t1));
+    x->stats.steps += 1;
+    x->stats.hits += *hit;
+    if (cont) { x->stats.steps_after_hit += 1; x->stats.ms_steps_cont += ms; }
+    else x->stats.ms_steps_fresh += ms;
+    x->stats.ms_decode += ms;
+    x->prev_hit = *hit != 0;
+    x->prev_b = b;
+    x->pos += 1;
+    x->pending = *token;
+    return PPD_OK;
+}
+
+int check_decode_args(ppd_ctx* x, int k, int l, int n) {
+    if (!x) return PPD_EINVAL;
+    if (!x->loaded || !x->prefilled) return PPD_ESTATE;
+    if (k < 0 || k > x->c.max_k || n < 0) return PPD_EINVAL;
+    if (k > 0 && (l < 1 || l > x->c.n_layers - 1)) return PPD_EINVAL;
+    // a PPD step touches position pos+1 (branch K/V commit)
+    if (x->pos + n + (k > 0 ? 1 : 0) > x->c.max_seq) return PPD_ENOSPC;
+    return PPD_OK;
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+
+extern "C" {
+
+size_t ppd_packed_bytes(int32_t n_rows, int32_t n_cols) {
+    if (n_rows < 1 || n_cols < 1) return 0;
+    return (size_t)((n_rows + kTileRows - 1) / kTileRows) * ((n_cols + kTileCols - 1) / kTileCols) * kTileBytes;
+}
+
+size_t ppd_device_bytes(const ppd_config* cfg) {
+    if (!valid_config(cfg)) return 0;
+    return plan(*cfg).total;
+}
+
+int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* stream_main, void* stream_branch,
+               ppd_ctx** out) {
+    if (!out) return PPD_EINVAL;
+    *out = nullptr;
+    if (!valid_config(cfg) || !dev_mem || ((uintptr_t)dev_mem % kAlign) != 0) return PPD_EINVAL;
+    if (!stream_main || !stream_branch || stream_main == stream_branch) return PPD_EINVAL;
+    Layout L = plan(*cfg);
+    if (dev_bytes < L.total) return PPD_ENOSPC;
+    ppd_ctx* x = new (std::nothrow) ppd_ctx();
+    if (!x) return PPD_EINVAL;
+    x->c = *cfg;
+    x->L = L;
+    x->base = reinterpret_cast<uint8_t*>(dev_mem);
+    x->sm = reinterpret_cast<cudaStream_t>(stream_main);
+    x->sb = reinterpret_cast<cudaStream_t>(stream_branch);
+    x->loaded = x->prefilled = false;
+    x->pdl = true;
+    x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
+    x->cuda_err = cudaSuccess;
+    std::memset(&x->stats, 0, sizeof(x->stats));
+    x->state = at<int>(x, L.state);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&x->ev_early, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&x->ev_branch, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreate(&x->ev_t0);
+    if (e == cudaSuccess) e = cudaEventCreate(&x->ev_t1);
+    if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&x->h_last), 64, cudaHostAllocDefault);
+    // everything except the weights starts at zero (activation padding, tickets, state, KV)
+    if (e == cudaSuccess) e = cudaMemsetAsync(x->base + L.weights_end, 0, L.total - L.weights_end, x->sm);
+    if (e == cudaSuccess) {
+        std::vector<int> pt(L.n_pages);
+        for (int i = 0; i < L.n_pages; ++i) pt[i] = i;
+        e = cudaMemcpyAsync(x->base + L.page_table, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, x->sm);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(x->sm);
+    }
+    if (e == cudaSuccess) e = launch_rope_table(at<float2>(x, L.rope), cfg->max_seq, cfg->head_dim, (double)cfg->rope_theta, x->sm);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(x->sm);
+    if (e != cudaSuccess) {
+        delete x;
+        return PPD_ECUDA;
+    }
+    for (int w = 0; w < 2; ++w) {
+        uint8_t* ws = x->base + L.ws[w];
+        x->lane[w].h = reinterpret_cast<float*>(ws + L.ws_h);
+        x->lane[w].qkv = reinterpret_cast<float*>(ws + L.ws_qkv);
+        x->lane[w].attn = reinterpret_cast<float*>(ws + L.ws_attn);
+        x->lane[w].z = reinterpret_cast<float*>(ws + L.ws_z);
+        x->lane[w].partial = reinterpret_cast<float*>(ws + L.ws_part);
+        x->lane[w].tickets = reinterpret_cast<int*>(ws + L.ws_tick);
+    }
+    *out = x;
+    return PPD_OK;
+}
+
+void ppd_destroy(ppd_ctx* x) {
+    if (!x) return;
+    cudaStreamSynchronize(x->sm);
+    cudaStreamSynchronize(x->sb);
+    cudaEventDestroy(x->ev_early);
+    cudaEventDestroy(x->ev_branch);
+    cudaEventDestroy(x->ev_t0);
+    cudaEventDestroy(x->ev_t1);
+    cudaFreeHost(x->h_last);
+    delete x;
+}
+
+int ppd_load_weights(ppd_ctx* x, const void* host_blob, size_t bytes, int dtype) {
+    if (!x || !host_blob || (dtype != 0 && dtype != 1)) return PPD_EINVAL;
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    const size_t D = c.d_model, F = c.d_ffn, V = c.vocab;
+    const size_t es = dtype == 0 ? 4 : 2;
+    const size_t elems = V * D + (size_t)c.n_layers * (2 * D + 4 * D * D + 3 * F * D) + D + V * D;
+    if (bytes != elems * es) return PPD_EINVAL;
+    const bool f32 = dtype == 0;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(host_blob);
+    uint8_t* staging = x->base + L.staging;
+    CK(cudaMemsetAsync(x->base, 0, L.weights_end, x->sm));   // tile padding must be zero
+
+    // Streams one [rows][cols] tensor through the staging buffer in row chunks.
+    auto upload = [&](size_t rows, size_t cols, auto&& consume) -> cudaError_t {
+        const size_t max_rows = kStagingBytes / (cols * es);
+        for (size_t r0 = 0; r0 < rows; r0 += max_rows) {
+            const size_t nr = rows - r0 < max_rows ? rows - r0 : max_rows;
+            cudaError_t e = cudaMemcpyAsync(staging, src + r0 * cols * es, nr * cols * es, cudaMemcpyHostToDevice, x->sm);
+            if (e != cudaSuccess) return e;
+            e = consume(r0, nr);
+            if (e != cudaSuccess) return e;
+        }
+        src += rows * cols * es;
+        return cudaSuccess;
+    };
+    auto pack_into = [&](uint16_t* dst, size_t rows, size_t cols, int row_mul, int row_off) -> cudaError_t {
+        return upload(rows, cols, [&](size_t r0, size_t nr) {
+            return launch_pack(staging, f32, (int)nr, (int)cols, dst, row_mul, row_off + (int)r0 * row_mul, x->sm);
+        });
+    };
+    auto vec_into = [&](float* dst, size_t n) -> cudaError_t {
+        return upload(1, n, [&](size_t, size_t) { return launch_convert(staging, f32, dst, true, n, x->sm); });
+    };
+
+    CK(upload(V, D, [&](size_t r0, size_t nr) {
+        return launch_convert(staging, f32, at<uint16_t>(x, L.emb) + r0 * D, false, nr * D, x->sm);
+    }));
+    for (int l = 0; l < c.n_layers; ++l) {
+        uint8_t* lb = layer_block(x, l);
+        uint16_t* wqkv = reinterpret_cast<uint16_t*>(lb + L.off_wqkv);
+        CK(vec_into(reinterpret_cast<float*>(lb + L.off_g1), D));
+        CK(pack_into(wqkv, D, D, 1, 0));
+        CK(pack_into(wqkv, D, D, 1, (int)D));
+        CK(pack_into(wqkv, D, D, 1, 2 * (int)D));
+        CK(pack_into(reinterpret_cast<uint16_t*>(lb + L.off_wo), D, D, 1, 0));
+        CK(vec_into(reinterpret_cast<float*>(lb + L.off_g2), D));
+        CK(pack_into(reinterpret_cast<uint16_t*>(lb + L.off_wgu), F, D, 2, 0));   // gate rows -> even
+        CK(pack_into(reinterpret_cast<uint16_t*>(lb + L.off_wgu), F, D, 2, 1));   // up rows   -> odd
+        CK(pack_into(reinterpret_cast<uint16_t*>(lb + L.off_wd), D, F, 1, 0));
+    }
+    CK(vec_into(at<float>(x, L.g_final), D));
+    CK(pack_into(at<uint16_t>(x, L.w_head), V, D, 1, 0));
+    CK(cudaStreamSynchronize(x->sm));
+    x->loaded = true;
+    x->prefilled = false;
+    return PPD_OK;
+}
+
+int ppd_prefill(ppd_ctx* x, const int32_t* prompt, int32_t n_prompt) {
+    if (!x || !prompt || n_prompt < 1) return PPD_EINVAL;
+    if (!x->loaded) return PPD_ESTATE;
+    if (n_prompt > x->c.max_seq) return PPD_ENOSPC;
+    for (int i = 0; i < n_prompt; ++i)
+        if (prompt[i] < 0 || prompt[i] >= x->c.vocab) return PPD_EINVAL;
+    const Layout& L = x->L;
+    CK(cudaMemcpyAsync(x->base + L.prompt, prompt, (size_t)n_prompt * 4, cudaMemcpyHostToDevice, x->sm));
+    CK(cudaStreamSynchronize(x->sm));   // the host array may be reused by the caller
+    const int64_t launches = x->stats.kernel_launches;
+    for (int t = 0; t + 1 < n_prompt; ++t) {
+        CK(launch_embed(at<uint16_t>(x, L.emb), at<int>(x, L.prompt) + t, 1, x->c.d_model, x->lane[0].h, L.Dp, x->sm, x->pdl));
+        int rc = run_layers(x, 0, 1, 0, x->c.n_layers, nullptr, t, false, x->sm);
+        if (rc) return rc;
+    }
+    x->stats.kernel_launches = launches;   // counted for decode steps only
+    CK(launch_set_state(x->state + S_POS, n_prompt - 1, x->state + S_PENDING, prompt[n_prompt - 1], x->state + S_STEP, 0, x->sm));
+    CK(cudaMemcpyAsync(x->h_last, x->state + S_LAST_TOKEN, 3 * sizeof(int), cudaMemcpyDeviceToHost, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    if (x->h_last[2] != 0) return PPD_ETIMEOUT;
+    x->pos = n_prompt - 1;
+    x->pending = prompt[n_prompt - 1];
+    x->prev_hit = false;
+    x->prefilled = true;
+    return PPD_OK;
+}
+
+int ppd_greedy_step(ppd_ctx* x, int32_t* out_token) {
+    if (!out_token) return PPD_EINVAL;
+    int rc = check_decode_args(x, 0, 0, 1);
+    if (rc) return rc;
+    uint8_t hit;
+    return decode_step(x, 0, 0, out_token, &hit);
+}
+
+int ppd_decode(ppd_ctx* x, int32_t k, int32_t l, int32_t n_tokens, int32_t eos, int32_t* out_tokens, uint8_t* out_hit,
+               int32_t* out_n) {
+    if (!out_n || (n_tokens > 0 && (!out_tokens || !out_hit))) return PPD_EINVAL;
+    *out_n = 0;
+    int rc = check_decode_args(x, k, l, n_tokens);
+    if (rc) return rc;
+    x->stats.ms_decode = 0.0;
+    for (int s = 0; s < n_tokens; ++s) {
+        int32_t tok;
+        uint8_t hit;
+        rc = decode_step(x, k, l, &tok, &hit);
+        if (rc) return rc;
+        out_tokens[s] = tok;
+        out_hit[s] = hit;
+        *out_n = s + 1;
+        if (eos >= 0 && tok == eos) break;
+    }
+    return PPD_OK;
+}
+
+int ppd_step(ppd_ctx* x, int32_t k, int32_t l, const int32_t* in_token, int32_t* out_token, uint8_t* out_hit) {
+    if (!out_token || !out_hit) return PPD_EINVAL;
+    int rc = check_decode_args(x, k, l, 1);
+    if (rc) return rc;
+    if (in_token) {
+        if (*in_token < 0 || *in_token >= x->c.vocab) return PPD_EINVAL;
+        CK(cudaMemcpyAsync(x->state + S_PENDING, in_token, 4, cudaMemcpyHostToDevice, x->sm));
+        if (*in_token != x->pending) x->prev_hit = false;
+        x->pending = *in_token;
+    }
+    return decode_step(x, k, l, out_token, out_hit);
+}
+
+int ppd_rewind(ppd_ctx* x, int32_t pos, int32_t pending_token) {
+    if (!x || pos < 0 || pos >= x->c.max_seq || pending_token < 0 || pending_token >= x->c.vocab) return PPD_EINVAL;
+    if (!x->loaded || !x->prefilled) return PPD_ESTATE;
+    if (pos > x->pos) return PPD_EINVAL;
+    CK(launch_set_state(x->state + S_POS, pos, x->state + S_PENDING, pending_token, x->state + S_STEP, 0, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    x->pos = pos;
+    x->pending = pending_token;
+    x->prev_hit = false;
+    return PPD_OK;
+}
+
+int32_t ppd_position(const ppd_ctx* x) { return x ? x->pos : -1; }
+
+int ppd_get_stats(ppd_ctx* x, ppd_stats* out) {
+    if (!x || !out) return PPD_EINVAL;
+    *out = x->stats;
+    return PPD_OK;
+}
+
+int ppd_reset_stats(ppd_ctx* x) {
+    if (!x) return PPD_EINVAL;
+    std::memset(&x->stats, 0, sizeof(x->stats));
+    return PPD_OK;
+}
+
+int ppd_debug_logits(ppd_ctx* x, float* final_logits, float* early_logits) {
+    if (!x) return PPD_EINVAL;
+    if (!x->prefilled) return PPD_ESTATE;
+    const size_t n = (size_t)x->c.vocab * 4;
+    if (final_logits) CK(cudaMemcpyAsync(final_logits, x->base + x->L.logits_final, n, cudaMemcpyDeviceToHost, x->sm));
+    if (early_logits) CK(cudaMemcpyAsync(early_logits, x->base + x->L.logits_early, n, cudaMemcpyDeviceToHost, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    return PPD_OK;
+}
+
+int ppd_debug_last(ppd_ctx* x, float* final_margin, int32_t* cand, int32_t k) {
+    if (!x || k < 0 || k > PPD_MAX_K) return PPD_EINVAL;
+    if (!x->prefilled) return PPD_ESTATE;
+    float vals[2];
+    CK(cudaMemcpyAsync(vals, at<float>(x, x->L.top_final) + 32, 8, cudaMemcpyDeviceToHost, x->sm));
+    if (cand && k > 0) CK(cudaMemcpyAsync(cand, x->base + x->L.top_early, (size_t)k * 4, cudaMemcpyDeviceToHost, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    if (final_margin) *final_margin = vals[0] - vals[1];
+    return PPD_OK;
+}
+
+int ppd_debug_force_token(ppd_ctx* x, int32_t token) {
+    if (!x || token < 0 || token >= x->c.vocab) return PPD_EINVAL;
+    if (!x->prefilled) return PPD_ESTATE;
+    CK(launch_set_state(nullptr, 0, x->state + S_PENDING, token, nullptr, 0, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    x->pending = token;
+    x->prev_hit = false;
+    return PPD_OK;
+}
+
+int ppd_debug_set_page_table(ppd_ctx* x, const int32_t* table, int32_t n_pages) {
+    if (!x || !table || n_pages != x->L.n_pages) return PPD_EINVAL;
+    if (x->prefilled) return PPD_ESTATE;
+    std::vector<char> seen(n_pages, 0);
+    for (int i = 0; i < n_pages; ++i) {
+        if (table[i] < 0 || table[i] >= n_pages || seen[table[i]]) return PPD_EINVAL;
+        seen[table[i]] = 1;
+    }
+    CK(cudaMemcpyAsync(x->base + x->L.page_table, table, (size_t)n_pages * 4, cudaMemcpyHostToDevice, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    return PPD_OK;
+}
+
+const char* ppd_strerror(int code) {
+    switch (code) {
+        case PPD_OK: return "ok";
+        case PPD_EINVAL: return "invalid argument";
+        case PPD_ENOSPC: return "KV cache or device arena too small";
+        case PPD_ESTATE: return "call out of order (load weights and prefill first)";
+        case PPD_ECUDA: return "CUDA error";
+        case PPD_ETIMEOUT: return "a bounded device-side wait gave up";
+    }
+    return "unknown error";
+}
+
+const char* ppd_last_cuda_error(const ppd_ctx* x) { return x ? cudaGetErrorString(x->cuda_err) : "no context"; }
+
+// ---------------------------------------------------------------- single operations
+
+#define CKOP(expr) do { if ((expr) != cudaSuccess) return PPD_ECUDA; } while (0)
+
+int ppd_op_pack(const uint16_t* src, int32_t n_src_rows, int32_t n_cols, void* dst, int32_t n_dst_rows, int32_t row_mul,
+                int32_t row_off, void* stream) {
+    if (!src || !dst || n_src_rows < 1 || n_cols < 1 || row_mul < 1 || row_off < 0) return PPD_EINVAL;
+    if ((long long)(n_src_rows - 1) * row_mul + row_off >= n_dst_rows) return PPD_EINVAL;
+    CKOP(launch_pack(src, false, n_src_rows, n_cols, reinterpret_cast<uint16_t*>(dst), row_mul, row_off,
+                     reinterpret_cast<cudaStream_t>(stream)));
+    return PPD_OK;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 1;
+    }
+    return n;
+}
+
+int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, const float* gain,
+                float eps, int32_t mode, const float* resid, float* out, int32_t ldo, void* stream) {
+    if (!w_packed || !x || !out || N < 1 || K < 1 || M < 1 || M > kMaxRows) return PPD_EINVAL;
+    if (mode < 0 || mode > 2 || (mode == 1 && !resid) || (mode == 2 && (N & 1))) return PPD_EINVAL;
+    if (ldx % kTileCols || ldx < round_up(K, kTileCols) || ldo < (mode == 2 ? N / 2 : N)) return PPD_EINVAL;
+    GemvArgs g{};
+    g.w = reinterpret_cast<const uint16_t*>(w_packed); g.N = N; g.K = K; g.x = x; g.ldx = ldx; g.gain = gain; g.eps = eps;
+    g.resid = resid; g.out = out; g.ldo = ldo; g.err = nullptr;
+    CKOP(launch_gemv(g, M, mode, reinterpret_cast<cudaStream_t>(stream), false, sm_count()));
+    return PPD_OK;
+}
+
+size_t ppd_op_head_scratch_bytes(void) { return kHeadScratchBytes + 2 * kMaxRows * 8 * 4; }
+
+int ppd_op_head_topk(const void* w_packed, int32_t vocab, int32_t K, const float* x, int32_t M, int32_t ldx,
+                     const float* gain, float eps, int32_t k, void* scratch, float* logits, int32_t* top_ids,
+                     float* top_vals, void* stream) {
+    if (!w_packed || !x || !scratch || !logits || !top_ids || !top_vals) return PPD_EINVAL;
+    if (vocab < 8 || K < 1 || M < 1 || M > kMaxRows || k < 1 || k > PPD_MAX_K) return PPD_EINVAL;
+    if (ldx % kTileCols || ldx < round_up(K, kTileCols)) return PPD_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // top-8 lists live behind the merge scratch; the first k of each row are copied out
+    int* ids8 = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) + kHeadScratchBytes);
+    float* vals8 = reinterpret_cast<float*>(ids8 + kMaxRows * 8);
+    GemvArgs g{};
+    g.w = reinterpret_cast<const uint16_t*>(w_packed); g.N = vocab; g.K = K; g.x = x; g.ldx = ldx; g.gain = gain; g.eps = eps;
+    g.out = logits; g.ldo = vocab; g.err = nullptr; g.head_scratch = scratch; g.top_ids = ids8; g.top_vals = vals8;
+    CKOP(launch_gemv(g, M, kHead, st, false, sm_count()));
+    CKOP(cudaMemcpy2DAsync(top_ids, (size_t)k * 4, ids8, 32, (size_t)k * 4, M, cudaMemcpyDeviceToDevice, st));
+    CKOP(cudaMemcpy2DAsync(top_vals, (size_t)k * 4, vals8, 32, (size_t)k * 4, M, cudaMemcpyDeviceToDevice, st));
+    return PPD_OK;
+}
+
+size_t ppd_op_attn_scratch_bytes(int32_t M, int32_t n_heads, int32_t head_dim, int32_t n_positions) {
+    if (M < 1 || n_heads < 1 || head_dim < 1 || n_positions < 1) return 0;
+    const int splits = (n_positions + kPageTokens - 1) / kPageTokens;
+    return align_up(attn_partial_floats(M, n_heads, head_dim, splits) * 4, kAlign) + align_up((size_t)n_heads * 4, kAlign);
+}
+
+int ppd_op_rope_table(float* table, int32_t n_positions, int32_t head_dim, float theta, void* stream) {
+    if (!table || n_positions < 1 || head_dim < 2 || (head_dim & 1)) return PPD_EINVAL;
+    CKOP(launch_rope_table(reinterpret_cast<float2*>(table), n_positions, head_dim, (double)theta,
+                           reinterpret_cast<cudaStream_t>(stream)));
+    return PPD_OK;
+}
+
+int ppd_op_attention(const float* qkv, int32_t M, int32_t n_heads, int32_t head_dim, int32_t n_prefix, void* kv_pages,
+                     const int32_t* page_table, void* branch_slots, const float* rope_table, void* scratch, float* out,
+                     int32_t ldo, void* stream) {
+    if (!qkv || !kv_pages || !page_table || !rope_table || !scratch || !out) return PPD_EINVAL;
+    if (M < 1 || M > kMaxRows || n_heads < 1 || (head_dim != 64 && head_dim != 128) || n_prefix < 0) return PPD_EINVAL;
+    if (ldo < n_heads * head_dim) return PPD_EINVAL;
+    const int splits = (n_prefix + 1 + kPageTokens - 1) / kPageTokens;
+    AttnArgs a{};
+    a.qkv = qkv; a.M = M; a.H = n_heads; a.hd = head_dim; a.d_pos = nullptr; a.pos_off = n_prefix;
+    a.kv_layer = reinterpret_cast<uint16_t*>(kv_pages); a.page_table = page_table;
+    a.slots = reinterpret_cast<uint16_t*>(branch_slots); a.slot_stride = 2ll * n_heads * head_dim;
+    a.rope = reinterpret_cast<const float2*>(rope_table);
+    a.partial = reinterpret_cast<float*>(scratch); a.max_splits = splits;
+    a.tickets = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) +
+                                       align_up(attn_partial_floats(M, n_heads, head_dim, splits) * 4, kAlign));
+    a.out = out; a.ldo = ldo; a.err = nullptr;
+    CKOP(launch_attention(a, reinterpret_cast<cudaStream_t>(stream), false, sm_count()));
+    return PPD_OK;
+}
+
+}  // extern "C"
