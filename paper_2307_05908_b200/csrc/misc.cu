@@ -54,13 +54,15 @@ cudaError_t launch_pack(const void* src, bool src_f32, int n_rows, int n_cols, u
     return cudaGetLastError();
 }
 
-// plain conversion to float32 (norm gains) or to bf16 bits (embedding table)
+// conversion of bf16 / float32 sources to bf16 values held as float32 (norm gains) or as bf16 bits (embedding table)
 template <bool SRC_F32, bool DST_F32>
 __global__ void convert_kernel(const void* __restrict__ src, void* __restrict__ dst, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         if (DST_F32) {
-            reinterpret_cast<float*>(dst)[i] = SRC_F32 ? reinterpret_cast<const float*>(src)[i]
-                                                       : bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(src)[i]);
+            // float32 sources are rounded to bf16 first: every parameter is a bf16 value
+            reinterpret_cast<float*>(dst)[i] =
+                bf16_bits_to_f32(SRC_F32 ? f32_to_bf16_bits(reinterpret_cast<const float*>(src)[i])
+                                         : reinterpret_cast<const uint16_t*>(src)[i]);
         } else {
             reinterpret_cast<uint16_t*>(dst)[i] = SRC_F32 ? f32_to_bf16_bits(reinterpret_cast<const float*>(src)[i])
                                                           : reinterpret_cast<const uint16_t*>(src)[i];

@@ -578,8 +578,8 @@ int ppd_debug_force_token(ppd_ctx* x, int32_t token) {
     if (!x->prefilled) return PPD_ESTATE;
     CK(launch_set_state(nullptr, 0, x->state + S_PENDING, token, nullptr, 0, x->sm));
     CK(cudaStreamSynchronize(x->sm));
+    if (token != x->pending) x->prev_hit = false;   // a committed branch belongs to the old token
     x->pending = token;
-    x->prev_hit = false;
     return PPD_OK;
 }
 
