@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the PPD decode path on B200.
+
+A "step" is one PPD decode step (one generated token): main pass through all layers, early head
+at layer l, k candidate branches overlapped with the main tail, final head, verify/commit.
+The default workload is the 7B-shaped random-init model, prompt 512, k = 3 at layer 16.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b|7b-long|13b|tiny]
+  python bench.py --impl reference ...      # the CPU oracle timed on the host cores
+
+Prints one JSON line.  With N > 1 (torchrun) every rank decodes its own replica (the path does
+not shard: batch 1 on one GPU); the line reports the slowest rank.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import ppd_inputs  # noqa: E402
+
+METRIC = "PPD ms/token (batch 1, 1 B200), with speedup vs greedy and HBM GB/s vs peak"
+UNIT = "ms/token"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ algorithmic bytes / flops
+
+def layer_bytes(s):
+    return 2 * (4 * s.d_model * s.d_model + 3 * s.d_ffn * s.d_model)
+
+
+def head_bytes(s):
+    return 2 * s.vocab * s.d_model
+
+
+def kv_layer_bytes(s, ctx_len):
+    return 2 * s.d_model * 2 * ctx_len          # K and V, bf16
+
+
+def greedy_step_bytes(s, ctx_len):
+    return s.n_layers * (layer_bytes(s) + kv_layer_bytes(s, ctx_len)) + head_bytes(s)
+
+
+def ppd_step_bytes(s, ctx_len, l, after_hit):
+    b = min(l, s.n_layers - l)
+    main_layers = s.n_layers - b if after_hit else s.n_layers
+    return ((main_layers + b) * (layer_bytes(s) + kv_layer_bytes(s, ctx_len)) + 2 * head_bytes(s))
+
+
+def ppd_step_flops(s, ctx_len, k, l, after_hit):
+    b = min(l, s.n_layers - l)
+    per_row_layer = layer_bytes(s) + 4 * s.d_model * ctx_len     # 2 flops per bf16 weight; attention 4*D*ctx
+    main_layers = s.n_layers - b if after_hit else s.n_layers
+    return (main_layers + k * b) * per_row_layer + 2 * head_bytes(s)
+
+
+def greedy_step_flops(s, ctx_len):
+    return s.n_layers * (layer_bytes(s) + 4 * s.d_model * ctx_len) + head_bytes(s)
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+
+        def num(x):
+            try:
+                return float(x)
+            except ValueError:
+                return None
+        sm = [num(r[0]) for r in rows if num(r[0]) is not None]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": num(rows[0][1]),
+                "power_w_max": max((num(r[2]) or 0) for r in rows), "samples": len(rows), "reasons": reasons}
+
+
+# ------------------------------------------------------------------ CPU oracle leg
+
+def oracle_sample(shape, k, l_full, n_steps, layers_sample=4):
+    """Times the oracle on a bounded sample: PPD on the first `layers_sample` layers of the model
+    (early layer at half of them), short prompt; scales per-layer and per-head times to full depth."""
+    from oracle import Oracle
+    sub = shape.with_layers(layers_sample)
+    blob = ppd_inputs.gen_weights(sub, seed=0)
+    prompt = ppd_inputs.gen_prompt(sub.vocab, 8, seed=1)
+    o = Oracle(sub, blob, max_seq=8 + n_steps + 2, max_k=k)
+    o.prefill(prompt)
+    tl0, th0 = o.times()
+    t0 = time.time()
+    r = o.ppd(n_steps, k, layers_sample // 2)
+    wall = time.time() - t0
+    tl1, th1 = o.times()
+    o.close()
+    ls = layers_sample // 2
+    bs = min(ls, layers_sample - ls)
+    hits_prev = int(r["hit"][:-1].sum())
+    layer_passes = n_steps * (layers_sample + k * bs) - hits_prev * bs
+    u = (tl1 - tl0) / layer_passes            # seconds per layer pass (one row)
+    e = (th1 - th0) / (2 * n_steps)           # seconds per head
+    d, b = shape.n_layers, min(l_full, shape.n_layers - l_full)
+    ppd_ms = 1e3 * ((d + k * b) * u + 2 * e)  # a step after a miss: nothing runs in parallel on the CPU
+    greedy_ms = 1e3 * (d * u + e)
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    sample = (f"oracle PPD k={k} on the first {layers_sample} of {d} layers (early layer {ls}), prompt 8, "
+              f"{n_steps} steps in {wall:.1f} s; per-layer {1e3 * u:.1f} ms and per-head {1e3 * e:.1f} ms scaled to "
+              f"(d + k*b) layers + 2 heads")
+    return {"value": ppd_ms, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+            "greedy_ms_per_token": greedy_ms, "sample_wall_s": wall}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # K steps + W warm-up steps of the truncated sample; one oracle call each so that exactly K are timed
+    cb = oracle_sample(wl.shape, args.k, args.l, max(args.warmup, 1))
+    cb = oracle_sample(wl.shape, args.k, args.l, args.steps)
+    line = {"metric": METRIC, "value": cb["value"], "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": cb["value"], "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(args, wl), "k": args.k, "early_layer": args.l},
+            "cpu_baseline": {k_: cb[k_] for k_ in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_name(args, wl):
+    return (f"{wl.shape.name}-shaped random-init bf16 (d={wl.shape.n_layers}, D={wl.shape.d_model}, F={wl.shape.d_ffn}, "
+            f"V={wl.shape.vocab}), prompt {args.prompt}, PPD k={args.k} at layer {args.l}, batch 1")
+
+
+# ------------------------------------------------------------------ GPU leg
+
+def time_kernel_gateup(ppd, torch, shape, stream, reps=3):
+    """Dominant kernel: fused RMSNorm + gate/up product + SwiGLU for one row.  Launched back to back
+    over 12 distinct weight matrices (larger than L2 together), timed with events on its stream."""
+    D, F = shape.d_model, shape.d_ffn
+    n_mats = 12
+    nbytes = ppd.packed_bytes(2 * F, D)
+    w = torch.empty(n_mats, nbytes, dtype=torch.uint8, device="cuda")
+    src = (torch.randn(1 << 22, device="cuda") * 0.02).bfloat16().view(torch.int16)
+    for i in range(n_mats):      # valid bf16 numbers; the content does not matter for timing
+        flat = w[i].view(torch.int16)
+        flat.copy_(src.repeat((flat.numel() + src.numel() - 1) // src.numel())[: flat.numel()])
+    x = torch.randn(1, (D + 255) // 256 * 256, device="cuda")
+    gain = torch.ones((D + 255) // 256 * 256, device="cuda")
+    out = torch.zeros(1, (F + 255) // 256 * 256, device="cuda")
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for i in range(n_mats):
+            ppd.op_gemv(w[i], 2 * F, D, x, gain, 1e-5, 2, None, out, stream=stream)
+        e0.record(stream)
+        for _ in range(reps):
+            for i in range(n_mats):
+                ppd.op_gemv(w[i], 2 * F, D, x, gain, 1e-5, 2, None, out, stream=stream)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / (reps * n_mats)
+    algo = 2 * F * D * 2 + D * 4 * 2 + F * 4          # weights + input row + gain + output
+    return ms, algo
+
+
+def run_gpu(args, wl):
+    import torch
+    import paper_2307_05908_b200 as ppd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the PPD path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    s, k, l, K, W, P = wl.shape, args.k, args.l, args.steps, args.warmup, args.prompt
+    blob = ppd_inputs.gen_weights(s, seed=0)
+    prompt = ppd_inputs.gen_prompt(s.vocab, P, seed=1)
+    ctx = ppd.Context(s, max_seq=P + W + K + 8, max_k=max(k, 1), device=f"cuda:{local}")
+    ctx.load_weights(blob)
+    del blob
+    ctx.prefill(prompt)
+    start_pos, start_tok = P - 1, int(prompt[-1])
+    stream = ctx.stream_main
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, tag):
+        """W warm-up steps, then K timed steps bracketed by events on the launching stream."""
+        ctx.rewind(start_pos, start_tok)
+        fn(W)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ctx.reset_stats()
+        t0 = time.time()
+        torch.cuda.nvtx.range_push(tag)       # lets a profiler select the timed region
+        e0.record(stream)
+        out = fn(K)
+        e1.record(stream)
+        barrier()
+        torch.cuda.nvtx.range_pop()
+        return e0.elapsed_time(e1), out, ctx.stats(), (t0, time.time())
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    ppd_ms, (tokens, hit), st_ppd, window = timed(lambda n: ctx.decode(k, l, n), "ppd_timed")
+    clocks = sampler.stop(*window)
+    greedy_ms, (gtokens, _), st_greedy, _ = timed(lambda n: ctx.decode(0, 0, n), "greedy_timed")
+    exact = bool((tokens == gtokens).all())
+
+    # end to end: host in the loop, the token crosses PCIe both ways every step
+    pinned = torch.empty(1, dtype=torch.int32).pin_memory()
+    pin_np = pinned.numpy()
+
+    def e2e_loop(n):
+        tok = None
+        for _ in range(n):
+            if tok is not None:
+                pin_np[0] = tok
+            tok, _ = ctx.step(k, l, pin_np if tok is not None else None)
+        return tok
+    ctx.rewind(start_pos, start_tok)
+    e2e_loop(W)
+    barrier()
+    t0 = time.perf_counter()
+    e2e_loop(K)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+
+    if dist is not None:
+        t = torch.tensor([ppd_ms, greedy_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ppd_ms, greedy_ms, e2e_ms = t.tolist()
+
+    peak, peak_kind = measured_peaks()
+    ctx_mid = P + W + K // 2
+    n_hit_prev = int(hit[:-1].sum())
+    frac_cont = n_hit_prev / max(K - 1, 1)
+    b = min(l, s.n_layers - l)
+    bytes_ppd = ((K - n_hit_prev) * ppd_step_bytes(s, ctx_mid, l, False) + n_hit_prev * ppd_step_bytes(s, ctx_mid, l, True)) / K
+    flops_ppd = ((K - n_hit_prev) * ppd_step_flops(s, ctx_mid, k, l, False) + n_hit_prev * ppd_step_flops(s, ctx_mid, k, l, True)) / K
+    bytes_greedy = greedy_step_bytes(s, ctx_mid)
+    ppd_tok_ms, greedy_tok_ms = ppd_ms / K, greedy_ms / K
+    t_fresh = st_ppd.ms_steps_fresh / max(st_ppd.steps - st_ppd.steps_after_hit, 1)
+    t_cont = st_ppd.ms_steps_cont / st_ppd.steps_after_hit if st_ppd.steps_after_hit else None
+    p_hat = float(hit.mean())
+    # the paper's latency model (Theorem 4.1) with measured step times, and in layer units
+    pred_ms = (K * t_fresh - (t_fresh - (t_cont if t_cont is not None else t_fresh)) * n_hit_prev) / K
+    breakeven = None
+    if t_cont is not None and t_fresh > t_cont:
+        breakeven = (t_fresh - greedy_tok_ms) / (t_fresh - t_cont) * K / max(K - 1, 1)
+
+    kern_ms, kern_bytes = time_kernel_gateup(ppd, torch, s, stream)
+    line = {
+        "metric": METRIC, "value": ppd_tok_ms, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ppd_tok_ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 accumulate on bf16 weights and bf16 KV", "data": "synthetic",
+        "config": {"workload": workload_name(args, wl), "k": k, "early_layer": l, "generate": K,
+                   "l2": "inputs larger than L2 (weights stream from HBM every step)",
+                   "replicas": world},
+        "tokens_per_s": 1e3 / ppd_tok_ms * world,
+        "greedy_ms_per_token": greedy_tok_ms, "greedy_tokens_per_s": 1e3 / greedy_tok_ms * world,
+        "speedup_vs_greedy": greedy_tok_ms / ppd_tok_ms,
+        "p_correct": p_hat, "ppd_equals_greedy": exact,
+        "ms_step_after_miss": t_fresh, "ms_step_after_hit": t_cont,
+        "predicted_ms_per_token_p_correct_model": pred_ms,
+        "paper_unit_prediction_ratio": 1 - (b / s.n_layers) * p_hat * (K - 1) / K,
+        "breakeven_p_correct": breakeven,
+        "bytes_per_token": {"greedy": bytes_greedy, "ppd": bytes_ppd, "extra": bytes_ppd - bytes_greedy},
+        "flops_per_token": {"greedy": greedy_step_flops(s, ctx_mid), "ppd": flops_ppd,
+                            "extra": flops_ppd - greedy_step_flops(s, ctx_mid)},
+        "step_roofline": {"bound": "hbm", "unit": "GB/s", "peak": peak, "peak_kind": peak_kind,
+                          "greedy_achieved": bytes_greedy / greedy_tok_ms / 1e6,
+                          "greedy_frac": bytes_greedy / greedy_tok_ms / 1e6 / peak,
+                          "ppd_achieved": bytes_ppd / ppd_tok_ms / 1e6, "ppd_frac": bytes_ppd / ppd_tok_ms / 1e6 / peak,
+                          "frac_steps_after_hit": frac_cont},
+        "roofline": {"bound": "hbm", "kernel": "gemv_kernel<1, swiglu, rmsnorm> (gate/up product)",
+                     "achieved": kern_bytes / kern_ms / 1e6, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": kern_bytes / kern_ms / 1e6 / peak, "traffic": None,
+                     "ms_per_launch": kern_ms, "algorithmic_bytes_per_launch": kern_bytes},
+        "e2e": {"value": e2e_ms / K, "unit": UNIT, "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 12},
+        "gpu_launches": int(st_ppd.kernel_launches),
+        "clocks": clocks,
+    }
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            cb = oracle_sample(s, k, l, 6)
+            line["cpu_baseline"] = {k_: cb[k_] for k_ in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b", choices=sorted(ppd_inputs.WORKLOADS))
+    ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--l", type=int, default=None)
+    ap.add_argument("--prompt", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="truncate the model to this many layers (small case for profiler captures)")
+    args = ap.parse_args()
+    wl = ppd_inputs.WORKLOADS[args.workload]
+    if args.layers:
+        import dataclasses
+        wl = dataclasses.replace(wl, shape=wl.shape.with_layers(args.layers), early_layer=max(1, args.layers // 2))
+    args.k = wl.k if args.k is None else args.k
+    args.l = wl.early_layer if args.l is None else args.l
+    args.prompt = wl.n_prompt if args.prompt is None else args.prompt
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_gpu(args, wl)
+
+
+if __name__ == "__main__":
+    main()
