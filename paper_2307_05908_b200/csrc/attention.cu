@@ -193,20 +193,46 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
     __syncthreads();
     if (!*flag) return;
     __threadfence();
-    if (tid < HD) {
-#pragma unroll
+    // Splits are merged in ascending order with the running-maximum recurrence.  The records of a
+    // row are contiguous ([split][HD+2]); they are staged through shared memory (the K/V tiles are
+    // idle now) in chunks, every thread keeping its loads in flight together, so a chunk costs
+    // about one L2 round trip.
+    {
+        constexpr int REC = HD + 2;
+        constexpr int CHUNK = (2 * S::kTile / 4) / REC;       // splits per chunk
+        constexpr int LPT = (CHUNK * REC + kAttnThreads - 1) / kAttnThreads;
+        float* stage = reinterpret_cast<float*>(smem + S::kKOff);
         for (int m = 0; m < M; ++m) {
-            const float* part = a.partial + ((size_t)m * H + h) * a.max_splits * (HD + 2);
-            float mx = __int_as_float(0xFF800000);
-            for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldcg(part + (size_t)s * (HD + 2) + HD));
-            float num = 0.f, den = 0.f;
-            for (int s = 0; s < n_splits; ++s) {
-                const float* ps = part + (size_t)s * (HD + 2);
-                const float w = exp2f(__ldcg(ps + HD) - mx);
-                num = fmaf(__ldcg(ps + tid), w, num);
-                den = fmaf(__ldcg(ps + HD + 1), w, den);
+            const float* part = a.partial + ((size_t)m * H + h) * a.max_splits * REC;
+            float mx = __int_as_float(0xFF800000), num = 0.f, den = 0.f;
+            for (int s0 = 0; s0 < n_splits; s0 += CHUNK) {
+                const int ns = min(CHUNK, n_splits - s0);
+                const int len = ns * REC;
+                float tmp[LPT];
+#pragma unroll
+                for (int j = 0; j < LPT; ++j) {
+                    const int c = tid + j * kAttnThreads;
+                    tmp[j] = c < len ? __ldcg(part + (size_t)s0 * REC + c) : 0.f;
+                }
+                __syncthreads();      // previous chunk fully consumed
+#pragma unroll
+                for (int j = 0; j < LPT; ++j) {
+                    const int c = tid + j * kAttnThreads;
+                    if (c < len) stage[c] = tmp[j];
+                }
+                __syncthreads();
+                if (tid < HD) {
+                    for (int s = 0; s < ns; ++s) {
+                        const float ms = stage[s * REC + HD];
+                        const float nm = fmaxf(mx, ms);
+                        const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
+                        num = fmaf(stage[s * REC + tid], wb, __fmul_rn(num, wa));
+                        den = fmaf(stage[s * REC + HD + 1], wb, __fmul_rn(den, wa));
+                        mx = nm;
+                    }
+                }
             }
-            a.out[(size_t)m * a.ldo + h * HD + tid] = num / den;
+            if (tid < HD) a.out[(size_t)m * a.ldo + h * HD + tid] = num / den;
         }
     }
     if (tid == 0) a.tickets[h] = 0;

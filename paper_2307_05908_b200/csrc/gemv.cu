@@ -299,15 +299,38 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvArgs a)
         consumer_sync();
         if (*flag) {
             __threadfence();
-            if (warp < M) {
-                float ov; int oi;
-                // the lists of row `warp` are contiguous: [ctas][8]
-                select8<true>(gv + (size_t)warp * kHeadMaxCtas * 8, gi + (size_t)warp * kHeadMaxCtas * 8, (int)gridDim.x * 8,
-                        lane, ov, oi);
-                if (lane < 8) {
-                    a.top_vals[warp * 8 + lane] = ov;
-                    a.top_ids[warp * 8 + lane] = oi;
+            // Stage each row's per-CTA lists into shared memory (the ring is idle by now) with all
+            // loads of a thread in flight at once, then select from shared memory: the merge costs
+            // about one L2 round trip instead of one per candidate.
+            float* sv = reinterpret_cast<float*>(smem);                  // [ctas*8] values
+            int* si = reinterpret_cast<int*>(smem) + kHeadMaxCtas * 8;   // [ctas*8] ids
+            const int n = (int)gridDim.x * 8;
+            for (int m = 0; m < M; ++m) {
+                const float* gvm = gv + (size_t)m * kHeadMaxCtas * 8;
+                const int* gim = gi + (size_t)m * kHeadMaxCtas * 8;
+                float tv[kHeadMaxCtas * 8 / 256];
+                int ti[kHeadMaxCtas * 8 / 256];
+#pragma unroll
+                for (int j = 0; j < kHeadMaxCtas * 8 / 256; ++j) {
+                    const int c = tid + j * 256;
+                    tv[j] = c < n ? __ldcg(gvm + c) : 0.f;
+                    ti[j] = c < n ? __ldcg(gim + c) : 0;
                 }
+#pragma unroll
+                for (int j = 0; j < kHeadMaxCtas * 8 / 256; ++j) {
+                    const int c = tid + j * 256;
+                    if (c < n) { sv[c] = tv[j]; si[c] = ti[j]; }
+                }
+                consumer_sync();
+                if (warp == 0) {
+                    float ov; int oi;
+                    select8<false>(sv, si, n, lane, ov, oi);
+                    if (lane < 8) {
+                        a.top_vals[m * 8 + lane] = ov;
+                        a.top_ids[m * 8 + lane] = oi;
+                    }
+                }
+                consumer_sync();
             }
             if (tid == 0) *ticket = 0;  // ready for the next launch
         }
