@@ -38,6 +38,7 @@ extern "C" {
 #define PPD_ESTATE (-3)   /* call out of order (decode before load/prefill)         */
 #define PPD_ECUDA (-4)    /* a CUDA call failed; see ppd_last_cuda_error            */
 #define PPD_ETIMEOUT (-5) /* a bounded device-side wait gave up; outputs are invalid */
+#define PPD_ELIMIT (-6)   /* a size exceeds a fixed capacity of the library            */
 
 #define PPD_MAX_K 8       /* largest supported number of early candidates            */
 
@@ -174,6 +175,27 @@ size_t ppd_op_head_scratch_bytes(void);
 int ppd_op_head_topk(const void* w_packed, int32_t vocab, int32_t K, const float* x, int32_t M,
                      int32_t ldx, const float* gain, float eps, int32_t k, void* scratch,
                      float* logits, int32_t* top_ids, float* top_vals, void* stream);
+
+/* The same head + top-k as ppd_op_head_topk for callers that cannot provide scratch memory.
+ * (The paper has no counterpart of this entry point; it exists for integration only.)
+ * Who needs it: code that may not allocate when it runs -- a plugin called while its host
+ * application has frozen the device heap, a worker whose memory pool was carved up at start-up,
+ * a latency-critical loop in which cudaMalloc is banned because it synchronises the device.
+ * Such a caller still passes its inputs and outputs, but the merge scratch (per-CTA candidate
+ * lists, arrival counter, merged lists: 132 KB) is a static device array inside the library
+ * image; every GPU that loads the library holds those 132 KB until the process exits.
+ *   - Limits: M <= 8 rows and k <= 8 candidates fit the array; larger values return PPD_ELIMIT
+ *     (device ordinals >= 64 too).  vocab and K are not limited by the scratch.
+ *   - This call never allocates or frees device memory.
+ *   - The first call on each device looks up the array's device address (one-time set-up with
+ *     that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     call re-zeroes the counter it needs on `stream`.  Two calls whose work overlaps on the
+ *     GPU (different streams, no ordering between them) race on the array: order them.
+ * Arguments and results are those of ppd_op_head_topk without `scratch`. */
+int ppd_op_head_topk_static(const void* w_packed, int32_t vocab, int32_t K, const float* x, int32_t M,
+                            int32_t ldx, const float* gain, float eps, int32_t k, float* logits,
+                            int32_t* top_ids, float* top_vals, void* stream);
 
 /* Decode attention for M query rows that share a cached prefix (Section 3: every process is fed
  * the same history x_<=t plus its own candidate).

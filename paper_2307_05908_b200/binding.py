@@ -16,7 +16,8 @@ from . import build as _build
 _LIB = None
 
 PPD_MAX_K = 8
-ERRORS = {0: "PPD_OK", -1: "PPD_EINVAL", -2: "PPD_ENOSPC", -3: "PPD_ESTATE", -4: "PPD_ECUDA", -5: "PPD_ETIMEOUT"}
+ERRORS = {0: "PPD_OK", -1: "PPD_EINVAL", -2: "PPD_ENOSPC", -3: "PPD_ESTATE", -4: "PPD_ECUDA", -5: "PPD_ETIMEOUT",
+          -6: "PPD_ELIMIT"}
 
 
 class PPDError(RuntimeError):
@@ -65,6 +66,7 @@ SIGNATURES = {
     "ppd_op_gemv": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _I, _P]),
     "ppd_op_head_scratch_bytes": (_SZ, []),
     "ppd_op_head_topk": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P, _P]),
+    "ppd_op_head_topk_static": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P]),
     "ppd_op_attn_scratch_bytes": (_SZ, [_I, _I, _I, _I]),
     "ppd_op_rope_table": (ctypes.c_int, [_P, _I, _I, _F, _P]),
     "ppd_op_attention": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _I, _P]),
@@ -251,6 +253,15 @@ def op_head_topk(w_packed, vocab, K, x, gain, eps, k, scratch, logits, top_ids, 
     _check(load().ppd_op_head_topk(w_packed.data_ptr(), vocab, K, x.data_ptr(), M, ldx,
                                    None if gain is None else gain.data_ptr(), eps, k, scratch.data_ptr(),
                                    logits.data_ptr(), top_ids.data_ptr(), top_vals.data_ptr(), _s(stream)))
+
+
+def op_head_topk_static(w_packed, vocab, K, x, gain, eps, k, logits, top_ids, top_vals, stream=None):
+    """Head + top-k whose scratch is a static device array of the library: the call allocates
+    nothing.  For callers that cannot allocate when they run; limits M <= 8, k <= 8."""
+    M, ldx = x.shape
+    _check(load().ppd_op_head_topk_static(w_packed.data_ptr(), vocab, K, x.data_ptr(), M, ldx,
+                                          None if gain is None else gain.data_ptr(), eps, k, logits.data_ptr(),
+                                          top_ids.data_ptr(), top_vals.data_ptr(), _s(stream)))
 
 
 def op_rope_table(table, n_positions, head_dim, theta, stream=None):

@@ -604,6 +604,7 @@ const char* ppd_strerror(int code) {
         case PPD_ESTATE: return "call out of order (load weights and prefill first)";
         case PPD_ECUDA: return "CUDA error";
         case PPD_ETIMEOUT: return "a bounded device-side wait gave up";
+        case PPD_ELIMIT: return "size beyond a fixed capacity of the library (static scratch: 8 rows, 8 candidates)";
     }
     return "unknown error";
 }

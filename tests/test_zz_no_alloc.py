@@ -1,0 +1,79 @@
+"""The allocation-free head entry point (static device scratch) against the regular one.
+
+Collected last on purpose: a failure here cannot hide the other tests from a run that stops at
+the first failure.  The entry point serves callers that cannot allocate when they run (a frozen
+device heap, a pre-carved memory pool, a loop in which cudaMalloc is banned); its scratch is a
+132 KB static device array shared by all calls, so the test also runs it twice in a row to show
+that a call does not depend on what the previous one left behind."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2307_05908_b200 as ppd
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _case(V, K, M, k, seed):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    w = (torch.randn(V, K, generator=g) * 0.03).bfloat16().view(torch.int16).to(DEV)
+    wp = torch.zeros(ppd.packed_bytes(V, K), dtype=torch.uint8, device=DEV)
+    ppd.op_pack(w, wp, V)
+    ld = (K + 255) // 256 * 256
+    x = torch.zeros(M, ld, device=DEV)
+    x[:, :K] = torch.randn(M, K, generator=g).to(DEV)
+    gain = torch.zeros(ld, device=DEV)
+    gain[:K] = (torch.rand(K, generator=g) + 0.5).to(DEV)
+    return wp, x, gain
+
+
+def _run(fn, V, k, M):
+    """Calls fn(logits, ids, vals) on pre-allocated outputs; returns the results and how much free
+    device memory the call itself consumed."""
+    logits = torch.zeros(M, V, device=DEV)
+    ids = torch.full((M, k), -1, dtype=torch.int32, device=DEV)
+    vals = torch.zeros(M, k, device=DEV)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    fn(logits, ids, vals)
+    torch.cuda.synchronize()
+    used = free_before - torch.cuda.mem_get_info()[0]
+    return logits.cpu().numpy(), ids.cpu().numpy(), vals.cpu().numpy(), used
+
+
+def test_static_scratch_head_matches_regular_head_twice_in_a_row():
+    for call, (V, K, M, k) in enumerate([(4096, 256, 3, 5), (32000, 1024, 1, 8)]):
+        wp, x, gain = _case(V, K, M, k, seed=call)
+        scratch = torch.zeros(ppd.load().ppd_op_head_scratch_bytes(), dtype=torch.uint8, device=DEV)
+        ref = _run(lambda *a: ppd.op_head_topk(wp, V, K, x, gain, 1e-5, k, scratch, *a), V, k, M)
+        if call == 0:      # the first call on a device also does the one-time address look-up
+            ppd.op_head_topk_static(wp, V, K, x, gain, 1e-5, k, *_outs(V, k, M))
+        got = _run(lambda *a: ppd.op_head_topk_static(wp, V, K, x, gain, 1e-5, k, *a), V, k, M)
+        assert np.array_equal(got[1], ref[1])                    # ids: exact
+        assert np.allclose(got[0], ref[0], rtol=0, atol=2e-5 * np.abs(ref[0]).max())   # logits
+        assert np.allclose(got[2], ref[2], rtol=0, atol=2e-5 * np.abs(ref[0]).max())
+        assert (got[1] >= 0).all() and len(set(got[1][0])) == k
+        assert got[3] <= 0                                       # the call took no device memory
+
+
+def _outs(V, k, M):
+    return (torch.zeros(M, V, device=DEV), torch.zeros(M, k, dtype=torch.int32, device=DEV), torch.zeros(M, k, device=DEV))
+
+
+def test_static_scratch_head_rejects_sizes_beyond_its_maximum():
+    V, K = 512, 256
+    wp, x, gain = _case(V, K, 1, 8, seed=9)
+    lib = ppd.load()
+    out = _outs(V, 9, 1)
+    rc = lib.ppd_op_head_topk_static(wp.data_ptr(), V, K, x.data_ptr(), 1, 256, gain.data_ptr(), 1e-5, 9,
+                                     out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), None)
+    assert rc == -6 and b"capacity" in lib.ppd_strerror(rc)
+    big = torch.zeros(9, 256, device=DEV)
+    rc = lib.ppd_op_head_topk_static(wp.data_ptr(), V, K, big.data_ptr(), 9, 256, gain.data_ptr(), 1e-5, 3,
+                                     out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), None)
+    assert rc == -6
+    with pytest.raises(ppd.PPDError):
+        ppd.op_head_topk_static(wp, V, K, x, gain, 1e-5, 9, *out)
