@@ -117,6 +117,14 @@ int ppd_rewind(ppd_ctx* ctx, int32_t pos, int32_t pending_token);
 /* Position of the pending token (= number of cached positions). */
 int32_t ppd_position(const ppd_ctx* ctx);
 
+/* Selects how a step is executed.  fused = 1 (default): one persistent kernel per step -- weights
+ * and cached K/V stream through one shared-memory ring across all layers, grid barriers separate
+ * the phases, and the k branch rows share each phase with the main row (the overlap of
+ * Algorithm 2's "in parallel" block).  fused = 0: one kernel per operation, main pass and branches
+ * on the two streams with events at the early head and before verify/commit.  Both give the same
+ * token stream as their own greedy decoding; logits of the two modes agree to rounding only. */
+int ppd_set_mode(ppd_ctx* ctx, int32_t fused);
+
 /* ---------------------------------------------------------------- inspection */
 
 int ppd_get_stats(ppd_ctx* ctx, ppd_stats* out);   /* out: host */
@@ -130,6 +138,11 @@ int ppd_debug_logits(ppd_ctx* ctx, float* final_logits, float* early_logits);
 int ppd_debug_last(ppd_ctx* ctx, float* final_margin, int32_t* cand, int32_t k);
 /* Replaces the pending token (teacher forcing for parity runs); drops any committed branch. */
 int ppd_debug_force_token(ppd_ctx* ctx, int32_t token);
+/* Phase timeline of the persistent step kernel (fused mode).  enable != 0 switches recording on
+ * for the following steps, 0 off.  If out != NULL, first copies the timestamps of the most recent
+ * traced step: out[(c * n_phases + p) * 2 + {0,1}] = start / end (ns, global timer) of phase p on
+ * CTA c (c = 0: first CTA, 1: last CTA); out: host, 4 * n_phases values; n_phases <= 512. */
+int ppd_debug_phase_times(ppd_ctx* ctx, int32_t enable, uint64_t* out, int32_t n_phases);
 /* Applies a permutation to the KV page table (host, n_pages entries, a permutation of
  * 0..n_pages-1, n_pages = ceil(max_seq / kv_page_tokens)); only valid right after create or
  * before prefill.  Exists to test that kernels honour the page table. */

@@ -53,12 +53,14 @@ SIGNATURES = {
     "ppd_step": (ctypes.c_int, [_P, _I, _I, _P, _P, _P]),
     "ppd_rewind": (ctypes.c_int, [_P, _I, _I]),
     "ppd_position": (_I, [_P]),
+    "ppd_set_mode": (ctypes.c_int, [_P, _I]),
     "ppd_get_stats": (ctypes.c_int, [_P, ctypes.POINTER(Stats)]),
     "ppd_reset_stats": (ctypes.c_int, [_P]),
     "ppd_debug_logits": (ctypes.c_int, [_P, _P, _P]),
     "ppd_debug_last": (ctypes.c_int, [_P, _P, _P, _I]),
     "ppd_debug_force_token": (ctypes.c_int, [_P, _I]),
     "ppd_debug_set_page_table": (ctypes.c_int, [_P, _P, _I]),
+    "ppd_debug_phase_times": (ctypes.c_int, [_P, _I, _P, _I]),
     "ppd_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "ppd_last_cuda_error": (ctypes.c_char_p, [_P]),
     "ppd_packed_bytes": (_SZ, [_I, _I]),
@@ -188,6 +190,11 @@ class Context:
         with self._dev():
             _check(self.lib.ppd_rewind(self._h, pos, int(pending_token)), self._h)
 
+    def set_mode(self, fused: bool):
+        """fused=True (default): one persistent kernel per step; False: per-op kernels on two streams."""
+        with self._dev():
+            _check(self.lib.ppd_set_mode(self._h, 1 if fused else 0), self._h)
+
     @property
     def position(self):
         return self.lib.ppd_position(self._h)
@@ -218,6 +225,15 @@ class Context:
     def force_token(self, token):
         with self._dev():
             _check(self.lib.ppd_debug_force_token(self._h, int(token)), self._h)
+
+    def phase_times(self, enable, n_phases=0):
+        """Switches the fused kernel's phase timeline on/off; returns the last traced step's
+        timestamps as a uint64 array [2 (first/last CTA)][n_phases][2 (start, end)] in ns."""
+        out = np.zeros((2, max(n_phases, 1), 2), dtype=np.uint64)
+        with self._dev():
+            _check(self.lib.ppd_debug_phase_times(self._h, 1 if enable else 0,
+                                                  out.ctypes.data if n_phases else None, n_phases), self._h)
+        return out[:, :n_phases]
 
     def set_page_table(self, table):
         t = np.ascontiguousarray(table, dtype=np.int32)

@@ -15,7 +15,7 @@ constexpr int kPageTokens = 64;      // KV positions per page
 constexpr int kMaxRows = 8;          // largest M (token rows per launch)
 
 // Device-side error word: 0 = fine; otherwise the code of the first wait that gave up.
-enum : int { kErrNone = 0, kErrFullWait = 1, kErrEmptyWait = 2, kErrKvWait = 3 };
+enum : int { kErrNone = 0, kErrFullWait = 1, kErrEmptyWait = 2, kErrKvWait = 3, kErrGridBarrier = 4, kErrPhaseWait = 5 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -66,9 +66,14 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* e
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3FFu) == 0 && global_timer_ns() - t0 > 2000000000ull) {
-            if (err) atomicCAS(err, 0, code);
-            return;
+        if ((++spins & 0x3FFu) == 0) {
+            const uint64_t waited = global_timer_ns() - t0;
+            // once some wait has already failed, the rest of the kernel only has to drain quickly
+            const bool failed_before = err && *reinterpret_cast<volatile int*>(err) != 0;
+            if (waited > 2000000000ull || (failed_before && waited > 1000000ull)) {
+                if (err) atomicCAS(err, 0, code);
+                return;
+            }
         }
     }
 }
@@ -81,6 +86,11 @@ __device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gmem_src, u
             smem_u32(smem_dst)),
         "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
+}
+
+// Asks L2 to fetch [p, p + bytes) from HBM without bringing it to the SM (fire and forget).
+__device__ __forceinline__ void bulk_prefetch_l2(const void* gmem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gmem_src), "r"(bytes) : "memory");
 }
 
 // ---- programmatic dependent launch
@@ -100,6 +110,30 @@ __device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {
     uint32_t u = __float_as_uint(f);
     u += 0x7FFFu + ((u >> 16) & 1u);
     return static_cast<uint16_t>(u >> 16);
+}
+
+// ---- packed pairs of floats (Blackwell executes fma/mul on two floats per instruction)
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// the two bf16 values of a 32-bit word as a packed pair of floats (element 2i low, 2i+1 high)
+__device__ __forceinline__ unsigned long long bf16x2_to_f32x2(uint32_t u) {
+    return pack2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -1,0 +1,1127 @@
+// Persistent decode-step kernel: a whole greedy step or a whole PPD step (Algorithm 2) in one
+// launch, one CTA per SM.
+//
+// The step is a sequence of phases separated by grid barriers: [embed] -> per layer {QKV, attention,
+// O, gate/up, down} -> early head -> branch embed -> fused layers {main layer l+i with 1 row  and
+// branch layer i with k rows in the same phase} -> final head -> verify/commit -> state update.
+// That is the paper's overlap of the k sub-processes with the main process's tail, expressed as
+// co-scheduled work of one persistent grid instead of separate processes.
+//
+// Everything that comes from HBM in bulk -- the packed weight tiles and the K/V pages of the
+// shared prefix -- flows through ONE shared-memory ring per CTA, filled by a producer thread with
+// bulk asynchronous copies (TMA) in program order.  The producer runs ahead of the consumers
+// across phase boundaries: the weights (and cached K/V) of the next phases are already on their
+// way while the grid barrier of the current phase resolves, so the HBM stream does not stop at
+// kernel or phase boundaries.  Only the small activation slices ("late" part of a stage) wait for
+// the phase to open.  Consumers never poll global memory: the producer polls the barrier counter
+// (bounded), then releases the late copies and signals a shared-memory barrier.
+//
+// Numerics: the same fixed per-row orders as the stand-alone kernels (a row's result does not
+// depend on how many rows share the launch), so PPD reproduces the greedy stream bit for bit.
+#include "common.cuh"
+#include "fused_step.cuh"
+#include "gemv.cuh"
+
+namespace ppd {
+namespace {
+
+constexpr int kCW = 8;                           // consumer warps
+constexpr int kThreads = (kCW + 2) * 32;     // + two producer warps (one thread of each is active)
+constexpr int kTS = 2;                           // weight tiles per stage
+constexpr int kStageW = kTS * kTileBytes;        // 32 KB: two weight tiles, or one K tile + one V tile
+constexpr int kRowX = kTS * kTileCols * 4;       // activation slice of one row in a stage (2 KB)
+constexpr int kMergeChunk = 16;                  // records merged per staging round
+constexpr int kUnitSplits = 16;                  // KV splits (pages) handled by one CTA for one head
+constexpr int kMaxSmem = 227 * 1024;
+
+enum PhaseKind : int {
+    PH_EMBED_MAIN = 0, PH_QKV = 1, PH_ATTN = 2, PH_O = 3, PH_GU = 4, PH_DOWN = 5,
+    PH_HEAD_EARLY = 6, PH_EMBED_BR = 7, PH_HEAD_FINAL = 8, PH_COMMIT = 9, PH_STATE = 10
+};
+
+template <int MB>
+struct Cfg {
+    static constexpr int MR = MB > 0 ? MB : 1;               // rows a stage can carry
+    static constexpr int kXOff = kStageW;
+    static constexpr int kGOff = kStageW + MR * kRowX;
+    static constexpr int kStageBytes = kGOff + kRowX;
+    // after the ring: barriers | union {attention warp states + merge staging, head merge staging} | head lists | flags
+    static constexpr int kBarBytes = 256;
+    static constexpr int kWs = 0;                                        // per-warp attention states [8 warps][MR][130] f32
+    static constexpr int kMerge = kWs + kCW * MR * 130 * 4;              // [kMergeChunk][130] f32
+    static constexpr int kUnionAttn = kMerge + kMergeChunk * 130 * 4;
+    static constexpr int kUnionHead = kHeadMaxCtas * 8 * 8;              // staged candidate lists
+    static constexpr int kUnion = ((kUnionAttn > kUnionHead ? kUnionAttn : kUnionHead) + 255) / 256 * 256;
+    static constexpr int kLists = kCW * kMaxRows * 8 * 8;                // per-warp top-8 lists
+    static constexpr int kFlags = 512;
+    static constexpr int kMisc = kBarBytes + kUnion + kLists + kFlags;
+    static constexpr int kStagesRaw = (kMaxSmem - kMisc) / kStageBytes;
+    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
+    static constexpr int kSmem = kStages * kStageBytes + kMisc;
+};
+
+struct Prog {
+    int mode, k, l, d, b, start, pos, la, n_seg_a, n_fused, embed_main, n_phases;
+};
+
+struct OpDesc {            // one matrix product of a phase, as seen by this CTA
+    const uint16_t* w;
+    const float* x;
+    const float* gain;
+    const float* resid;
+    float* out;
+    int N, K, n_rg, n_kc, spr, ldx, ldo, mode, M, first_rg;
+};
+
+struct AttnDesc {          // the attention work of one lane in a phase, as seen by this CTA
+    // A unit = (head, range of up to kUnitSplits consecutive KV pages); R units per head.
+    int M, p, n_splits, s_tail, R, units, first_unit;
+    const float* qkv;
+    uint16_t* kv_layer;
+    uint16_t* slots;       // this layer's slots (row m at + m*slot_stride) or nullptr = cache
+    float* out;
+    float* partial;
+    int* tickets;
+};
+
+struct PhaseDesc {
+    int kind, n_ops;
+    OpDesc op[2];
+    AttnDesc at[2];
+};
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+__device__ Prog build_prog(const FusedArgs& a) {
+    Prog P;
+    P.mode = a.mode; P.k = a.k; P.l = a.l; P.d = a.d;
+    P.b = 0; P.start = 0;
+    if (a.mode == kPrefillToken) {
+        P.pos = a.pos_val;
+    } else {
+        P.pos = __ldcg(a.state + S_POS);
+        const int prev_hit = __ldcg(a.state + S_PREV_HIT), prev_b = __ldcg(a.state + S_PREV_B);
+        if (a.mode == kPpdStep) P.b = a.l < a.d - a.l ? a.l : a.d - a.l;
+        // after a hit, layers 1..prev_b of the pending token were committed from its branch
+        if (prev_hit && !(a.mode == kPpdStep && prev_b > a.l)) P.start = prev_b;
+    }
+    P.la = a.mode == kPpdStep ? a.l : a.d;
+    P.n_seg_a = P.la - P.start;
+    P.n_fused = a.mode == kPpdStep ? a.d - a.l : 0;
+    P.embed_main = P.start == 0;
+    P.n_phases = P.embed_main + 5 * P.n_seg_a + (a.mode == kPpdStep ? 2 + 5 * P.n_fused : 0) +
+                 (a.mode != kPrefillToken ? 2 : 0) + 1;
+    return P;
+}
+
+__device__ void phase_info(const Prog& P, int ph, int& kind, int& lm, int& lb) {
+    lm = lb = -1;
+    int q = ph;
+    if (P.embed_main) {
+        if (q == 0) { kind = PH_EMBED_MAIN; return; }
+        --q;
+    }
+    if (q < 5 * P.n_seg_a) { kind = PH_QKV + q % 5; lm = P.start + q / 5; return; }
+    q -= 5 * P.n_seg_a;
+    if (P.mode == kPpdStep) {
+        if (q == 0) { kind = PH_HEAD_EARLY; return; }
+        if (q == 1) { kind = PH_EMBED_BR; return; }
+        q -= 2;
+        if (q < 5 * P.n_fused) {
+            kind = PH_QKV + q % 5;
+            const int i = q / 5;
+            lm = P.l + i;
+            lb = i < P.b ? i : -1;
+            return;
+        }
+        q -= 5 * P.n_fused;
+    }
+    if (P.mode != kPrefillToken) {
+        if (q == 0) { kind = PH_HEAD_FINAL; return; }
+        if (q == 1) { kind = PH_COMMIT; return; }
+    }
+    kind = PH_STATE;
+}
+
+__device__ void fill_op(const FusedArgs& a, int kind, int layer, const LaneBuf& ln, int M, int cta_off, OpDesc& o) {
+    const uint8_t* lb = a.layers + (size_t)layer * a.layer_bytes;
+    const int G = gridDim.x;
+    o.M = M;
+    o.resid = nullptr;
+    o.gain = nullptr;
+    switch (kind) {
+        case PH_QKV:
+            o.w = reinterpret_cast<const uint16_t*>(lb + a.off_wqkv); o.N = 3 * a.D; o.K = a.D;
+            o.x = ln.h; o.ldx = a.Dp; o.gain = reinterpret_cast<const float*>(lb + a.off_g1);
+            o.mode = kStore; o.out = ln.qkv; o.ldo = 3 * a.D;
+            break;
+        case PH_O:
+            o.w = reinterpret_cast<const uint16_t*>(lb + a.off_wo); o.N = a.D; o.K = a.D;
+            o.x = ln.attn; o.ldx = a.Dp; o.mode = kResid; o.resid = ln.h; o.out = ln.h; o.ldo = a.Dp;
+            break;
+        case PH_GU:
+            o.w = reinterpret_cast<const uint16_t*>(lb + a.off_wgu); o.N = 2 * a.F; o.K = a.D;
+            o.x = ln.h; o.ldx = a.Dp; o.gain = reinterpret_cast<const float*>(lb + a.off_g2);
+            o.mode = kSwiglu; o.out = ln.z; o.ldo = a.Fp;
+            break;
+        default:  // PH_DOWN
+            o.w = reinterpret_cast<const uint16_t*>(lb + a.off_wd); o.N = a.D; o.K = a.F;
+            o.x = ln.z; o.ldx = a.Fp; o.mode = kResid; o.resid = ln.h; o.out = ln.h; o.ldo = a.Dp;
+            break;
+    }
+    o.n_rg = (o.N + kTileRows - 1) / kTileRows;
+    o.n_kc = (o.K + kTileCols - 1) / kTileCols;
+    o.spr = (o.n_kc + kTS - 1) / kTS;
+    o.first_rg = ((int)blockIdx.x - cta_off + G) % G;
+}
+
+__device__ void fill_attn(const FusedArgs& a, int layer, const LaneBuf& ln, int M, int p, bool branch, int cta_off, AttnDesc& t) {
+    const int G = gridDim.x;
+    t.M = M; t.p = p;
+    t.n_splits = p / kPageTokens + 1;
+    t.s_tail = p / kPageTokens;
+    t.R = (t.n_splits + kUnitSplits - 1) / kUnitSplits;
+    t.units = a.H * t.R;
+    t.first_unit = ((int)blockIdx.x - cta_off + G) % G;
+    t.qkv = ln.qkv;
+    t.kv_layer = a.kv + (size_t)layer * a.kv_layer_elems;
+    t.slots = branch ? a.slots + (size_t)layer * a.slot_layer_stride : nullptr;
+    t.out = ln.attn; t.partial = ln.partial; t.tickets = ln.tickets;
+}
+
+__device__ void make_phase(const FusedArgs& a, const Prog& P, int ph, int MB, PhaseDesc& pd) {
+    int lm, lb;
+    phase_info(P, ph, pd.kind, lm, lb);
+    pd.n_ops = 0;
+    const int G = gridDim.x;
+    if (pd.kind == PH_QKV || pd.kind == PH_O || pd.kind == PH_GU || pd.kind == PH_DOWN) {
+        fill_op(a, pd.kind, lm, a.main, 1, 0, pd.op[0]);
+        pd.n_ops = 1;
+        if (lb >= 0) { fill_op(a, pd.kind, lb, a.br, MB, G / 2, pd.op[1]); pd.n_ops = 2; }
+    } else if (pd.kind == PH_ATTN) {
+        fill_attn(a, lm, a.main, 1, P.pos, false, 0, pd.at[0]);
+        pd.n_ops = 1;
+        if (lb >= 0) { fill_attn(a, lb, a.br, MB, P.pos + 1, true, G / 2, pd.at[1]); pd.n_ops = 2; }
+    } else if (pd.kind == PH_HEAD_EARLY || pd.kind == PH_HEAD_FINAL) {
+        OpDesc& o = pd.op[0];
+        o.w = a.w_head; o.N = a.V; o.K = a.D; o.x = a.main.h; o.ldx = a.Dp; o.gain = a.g_final; o.resid = nullptr;
+        o.mode = kHead; o.out = pd.kind == PH_HEAD_EARLY ? a.logits_early : a.logits_final; o.ldo = a.V; o.M = 1;
+        o.n_rg = (o.N + kTileRows - 1) / kTileRows;
+        o.n_kc = (o.K + kTileCols - 1) / kTileCols;
+        o.spr = (o.n_kc + kTS - 1) / kTS;
+        o.first_rg = blockIdx.x;
+        pd.n_ops = 1;
+    }
+}
+
+__device__ __forceinline__ bool phase_has_gemv(int kind) {
+    return kind == PH_QKV || kind == PH_O || kind == PH_GU || kind == PH_DOWN || kind == PH_HEAD_EARLY || kind == PH_HEAD_FINAL;
+}
+
+// ------------------------------------------------------------------------------------- producer
+
+struct Item {
+    int ph, kind, lane;
+    int rg, c0, nt;      // matrix stage
+    int h, s, n_valid;   // attention stage
+    bool tail;
+    bool kv_late;        // the K/V tile holds a position written earlier in this launch: no prefetch
+};
+
+// Calls f(phase descriptor, item) for every ring stage of this CTA, in program order: phases in
+// order; inside a phase the main lane's stages, then the branch lane's.  Producers and consumers
+// all walk this same order.
+template <typename F>
+__device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P, int MB, F&& f) {
+    const int G = gridDim.x;
+    PhaseDesc pd;
+    Item it;
+    for (int ph = 0; ph < P.n_phases; ++ph) {
+        int kind, lm, lb;
+        phase_info(P, ph, kind, lm, lb);
+        if (!phase_has_gemv(kind) && kind != PH_ATTN) continue;
+        make_phase(a, P, ph, MB, pd);
+        it.ph = ph;
+        it.kind = kind;
+        if (kind == PH_ATTN) {
+            for (int ln = 0; ln < pd.n_ops; ++ln) {
+                const AttnDesc& t = pd.at[ln];
+                it.lane = ln;
+                for (int u = t.first_unit; u < t.units; u += G) {
+                    it.h = u / t.R;
+                    const int s_lo = (u - it.h * t.R) * kUnitSplits, s_hi = min(t.n_splits, s_lo + kUnitSplits);
+                    for (int sp = s_lo; sp < s_hi; ++sp) {
+                        it.s = sp;
+                        it.n_valid = min(kPageTokens, t.p - sp * kPageTokens);
+                        it.tail = sp == t.s_tail;
+                        // a branch row's prefix ends with the position the main pass wrote in this launch
+                        it.kv_late = ln == 1 && sp == P.pos / kPageTokens;
+                        f(pd, it);
+                    }
+                }
+            }
+        } else {
+            for (int ln = 0; ln < pd.n_ops; ++ln) {
+                const OpDesc& o = pd.op[ln];
+                it.lane = ln;
+                for (int rg = o.first_rg; rg < o.n_rg; rg += G) {
+                    it.rg = rg;
+                    for (int c0 = 0; c0 < o.n_kc; c0 += kTS) {
+                        it.c0 = c0;
+                        it.nt = min(kTS, o.n_kc - c0);
+                        f(pd, it);
+                    }
+                }
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t item_bytes(const FusedArgs& a, const PhaseDesc& pd, const Item& it) {
+    if (it.kind == PH_ATTN) {
+        const AttnDesc& t = pd.at[it.lane];
+        return (it.n_valid > 0 ? 2u * kPageTokens * a.hd * 2 : 0u) + (uint32_t)t.M * a.hd * 4 * (it.tail ? 3 : 1);
+    }
+    const OpDesc& o = pd.op[it.lane];
+    return (uint32_t)it.nt * kTileBytes + (uint32_t)o.M * it.nt * kTileCols * 4 + (o.gain ? (uint32_t)it.nt * kTileCols * 4 : 0u);
+}
+
+__device__ __forceinline__ void issue_kv(const FusedArgs& a, const AttnDesc& t, const Item& it, uint8_t* st, uint64_t* full) {
+    const size_t page_elems = (size_t)2 * a.H * kPageTokens * a.hd;
+    const uint32_t tile = kPageTokens * a.hd * 2;
+    const uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + it.s) * page_elems + (size_t)it.h * kPageTokens * a.hd;
+    bulk_g2s(st, pg, tile, full);
+    bulk_g2s(st + tile, pg + (size_t)a.H * kPageTokens * a.hd, tile, full);
+}
+
+// bulk data that does not depend on the current step's activations: weights and cached K/V
+__device__ __forceinline__ void issue_early(const FusedArgs& a, const PhaseDesc& pd, const Item& it, uint8_t* st, uint64_t* full) {
+    mbar_arrive_expect_tx(full, item_bytes(a, pd, it));
+    if (it.kind == PH_ATTN) {
+        if (it.n_valid > 0 && !it.kv_late) issue_kv(a, pd.at[it.lane], it, st, full);
+    } else {
+        const OpDesc& o = pd.op[it.lane];
+        bulk_g2s(st, o.w + ((size_t)it.rg * o.n_kc + it.c0) * kTileElems, it.nt * kTileBytes, full);
+    }
+}
+
+// activation slices: only valid once the phase is open
+template <int MB>
+__device__ __forceinline__ void issue_late(const FusedArgs& a, const PhaseDesc& pd, const Item& it, uint8_t* st, uint64_t* full) {
+    using C = Cfg<MB>;
+    if (it.kind == PH_ATTN) {
+        const AttnDesc& t = pd.at[it.lane];
+        if (it.n_valid > 0 && it.kv_late) issue_kv(a, t, it, st, full);
+        const uint32_t row = a.hd * 4;
+        const int parts = it.tail ? 3 : 1;   // q, and for the tail split the new k and v rows
+        for (int part = 0; part < parts; ++part)
+            for (int m = 0; m < t.M; ++m)
+                bulk_g2s(st + C::kXOff + (part * t.M + m) * row, t.qkv + (size_t)m * 3 * a.D + part * a.D + it.h * a.hd, row, full);
+    } else {
+        const OpDesc& o = pd.op[it.lane];
+        for (int m = 0; m < o.M; ++m)
+            bulk_g2s(st + C::kXOff + m * kRowX, o.x + (size_t)m * o.ldx + (size_t)it.c0 * kTileCols, it.nt * kTileCols * 4, full);
+        if (o.gain) bulk_g2s(st + C::kGOff, o.gain + (size_t)it.c0 * kTileCols, it.nt * kTileCols * 4, full);
+    }
+}
+
+// Producer W (one thread): arms each stage and prefetches its weights / cached K/V as soon as the
+// ring slot is free; runs ahead of the consumers across phase boundaries.
+template <int MB>
+__device__ void producer_w(const FusedArgs& a, const Prog& P, uint8_t* smem, uint64_t* full, uint64_t* empty, volatile int* n_w_pub) {
+    using C = Cfg<MB>;
+    int* err = a.state + S_ERR;
+    int n_w = 0;
+    for_each_item(a, P, MB, [&](const PhaseDesc& pd, const Item& it) {
+        const int slot = n_w % C::kStages;
+        if (n_w >= C::kStages) mbar_wait(&empty[slot], ((n_w / C::kStages) - 1) & 1, err, kErrEmptyWait);
+        issue_early(a, pd, it, smem + slot * C::kStageBytes, &full[slot]);
+        ++n_w;
+        __threadfence_block();
+        *n_w_pub = n_w;
+    });
+}
+
+// Producer X (one thread): watches the grid-barrier counter, opens phases for the consumers, and
+// sends the activation slices of every armed stage whose phase is open.
+template <int MB>
+__device__ void producer_x(const FusedArgs& a, const Prog& P, uint8_t* smem, uint64_t* full, uint64_t* phase_bar, volatile int* n_w_pub) {
+    using C = Cfg<MB>;
+    const unsigned long long* cnt = reinterpret_cast<const unsigned long long*>(a.state + S_BAR_COUNT);
+    const unsigned long long base = __ldcg(reinterpret_cast<const unsigned long long*>(a.state + S_BAR_BASE));
+    const unsigned long long G = gridDim.x;
+    int* err = a.state + S_ERR;
+    int n_x = 0, open = 0;
+    uint64_t t_idle = 0;
+    mbar_arrive(phase_bar);   // phase 0: its inputs come from earlier kernels
+
+    // One look at the grid barrier; opens the next phase if every CTA has arrived.  Bounded: after
+    // ~2 s without any progress the error word is set and the phase is forced open so that every
+    // wait in the CTA ends and the kernel terminates (outputs are then invalid).
+    auto poll = [&]() {
+        if (open >= P.n_phases - 1) return;
+        bool opened = ld_acquire_u64(cnt) >= base + (unsigned long long)(open + 1) * G;
+        if (!opened) {
+            const uint64_t now = global_timer_ns();
+            if (t_idle == 0) t_idle = now;
+            else if (now - t_idle > 2000000000ull ||
+                     (*reinterpret_cast<volatile int*>(err) != 0 && now - t_idle > 1000000ull)) {
+                atomicCAS(err, 0, kErrGridBarrier);
+                opened = true;
+            }
+        }
+        if (opened) {
+            ++open;
+            t_idle = 0;
+            fence_proxy_async();
+            mbar_arrive(phase_bar);
+        }
+    };
+
+    for_each_item(a, P, MB, [&](const PhaseDesc& pd, const Item& it) {
+        while (it.ph > open) poll();
+        // wait until producer W has armed this stage; keep opening phases meanwhile (the consumers
+        // of a stage-less phase may be what frees the ring)
+        uint64_t t0 = 0;
+        while (n_x >= *n_w_pub) {
+            poll();
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 4000000000ull) { atomicCAS(err, 0, kErrEmptyWait); break; }
+        }
+        t_idle = 0;
+        const int slot = n_x % C::kStages;
+        issue_late<MB>(a, pd, it, smem + slot * C::kStageBytes, &full[slot]);
+        ++n_x;
+    });
+    while (open < P.n_phases - 1) poll();
+}
+
+// ------------------------------------------------------------------------------------- consumers
+
+struct Shared {
+    uint8_t* ring;
+    uint64_t *full, *empty, *phase_bar;
+    uint8_t* un;      // union region
+    float* lists_v;   // [8 rows][8 warps][8]
+    int* lists_i;
+    int* flags;
+};
+
+__device__ __forceinline__ void list_insert(float& lv, int& li, float nv, int ni, int lane) {
+    const unsigned ahead = __ballot_sync(0xFFFFFFFFu, lane < 8 && better(lv, li, nv, ni));
+    const int pos = __popc(ahead);
+    const float upv = __shfl_up_sync(0xFFFFFFFFu, lv, 1);
+    const int upi = __shfl_up_sync(0xFFFFFFFFu, li, 1);
+    if (lane < 8) {
+        if (lane > pos) { lv = upv; li = upi; }
+        else if (lane == pos) { lv = nv; li = ni; }
+    }
+}
+
+// the 8 best of n (value, id) pairs in shared memory, in total order, into lanes 0..7
+__device__ __forceinline__ void select8(const float* vals, const int* ids, int n, int lane, float& ov, int& oi) {
+    float pv = __int_as_float(0x7F800000);
+    int pi = -1;
+    ov = __int_as_float(0xFF800000);
+    oi = 0x7FFFFFFF;
+    for (int r = 0; r < 8; ++r) {
+        float bv = __int_as_float(0xFF800000);
+        int bi = 0x7FFFFFFF;
+        for (int c = lane; c < n; c += 32) {
+            const float v = vals[c];
+            const int i = ids[c];
+            if (better(pv, pi, v, i) && better(v, i, bv, bi)) { bv = v; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v2 = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+            const int i2 = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+            if (better(v2, i2, bv, bi)) { bv = v2; bi = i2; }
+        }
+        if (lane == r) { ov = bv; oi = bi; }
+        pv = bv; pi = bi;
+    }
+}
+
+// One matrix product: this CTA's row groups, stages taken from the ring in program order.
+// RMSNorm is applied as  y = (sum_k W[n][k] * (g[k] h[k])) / rms(h): the sum of squares is
+// gathered from the same slices while the first row group streams by, so no extra pass over h.
+template <int M, int MODE, bool NORM, int MB>
+__device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, float* lv, int* li) {
+    using C = Cfg<MB>;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x;
+    int* err = a.state + S_ERR;
+    const int r0 = warp * 4;
+    // Per (row of the batch, weight row): one packed accumulator {sum over even k, sum over odd k};
+    // a lane adds its four column pairs of every tile in a fixed order, the halves are added at the
+    // end, then the lanes are summed by a fixed shuffle tree.
+    float inv[M];
+    unsigned long long ssq[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) { inv[m] = 1.f; ssq[m] = 0ull; }
+    bool first = true;
+    for (int rg = op.first_rg; rg < op.n_rg; rg += G) {
+        unsigned long long acc2[M][4];
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc2[m][r] = 0ull;
+        for (int c0 = 0; c0 < op.n_kc; c0 += kTS, ++it) {
+            const int slot = it % C::kStages;
+            mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
+            const uint8_t* st = sh.ring + slot * C::kStageBytes;
+            const int nt = min(kTS, op.n_kc - c0);
+#pragma unroll
+            for (int t = 0; t < kTS; ++t) {
+                if (t < nt) {
+                    const uint4* wt = reinterpret_cast<const uint4*>(st + t * kTileBytes) + r0 * 32 + lane;
+                    uint4 w[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) w[r] = wt[r * 32];
+                    unsigned long long xv[M][4];
+                    unsigned long long gs[4];
+                    if (NORM) {
+                        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(st + C::kGOff) + t * (kTileCols / 4) + lane * 2;
+                        const ulonglong2 g0 = gp[0], g1 = gp[1];
+                        gs[0] = g0.x; gs[1] = g0.y; gs[2] = g1.x; gs[3] = g1.y;
+                    }
+#pragma unroll
+                    for (int m = 0; m < M; ++m) {
+                        const ulonglong2* xp = reinterpret_cast<const ulonglong2*>(st + C::kXOff + m * kRowX) + t * (kTileCols / 4) + lane * 2;
+                        const ulonglong2 x0 = xp[0], x1 = xp[1];
+                        xv[m][0] = x0.x; xv[m][1] = x0.y; xv[m][2] = x1.x; xv[m][3] = x1.y;
+                        if (NORM) {
+                            if (first) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) ssq[m] = ffma2(xv[m][j], xv[m][j], ssq[m]);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) xv[m][j] = fmul2(xv[m][j], gs[j]);
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        unsigned long long wf[4];
+                        wf[0] = bf16x2_to_f32x2(w[r].x); wf[1] = bf16x2_to_f32x2(w[r].y);
+                        wf[2] = bf16x2_to_f32x2(w[r].z); wf[3] = bf16x2_to_f32x2(w[r].w);
+#pragma unroll
+                        for (int m = 0; m < M; ++m)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) acc2[m][r] = ffma2(wf[j], xv[m][j], acc2[m][r]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+        }
+        if (NORM && first) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                float s0, s1;
+                unpack2(ssq[m], s0, s1);
+                inv[m] = 1.0f / sqrtf(warp_sum(s0 + s1) / (float)op.K + a.eps);
+            }
+        }
+        first = false;
+        float acc[M][4];
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                float s0, s1;
+                unpack2(acc2[m][r], s0, s1);
+                acc[m][r] = warp_sum(s0 + s1);
+                if (NORM) acc[m][r] = __fmul_rn(acc[m][r], inv[m]);
+            }
+        const int n0 = rg * kTileRows + r0;
+        if (MODE == kStore || MODE == kResid || MODE == kHead) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const float v = lane == 0 ? acc[m][0] : lane == 1 ? acc[m][1] : lane == 2 ? acc[m][2] : acc[m][3];
+                const int n = n0 + lane;
+                if (lane < 4 && n < op.N) {
+                    const size_t o = (size_t)m * op.ldo + n;
+                    op.out[o] = (MODE == kResid) ? __ldcg(op.resid + o) + v : v;
+                }
+                if (MODE == kHead) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+                        if (n0 + r < op.N) list_insert(lv[m], li[m], acc[m][r], n0 + r, lane);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const float g = lane == 0 ? acc[m][0] : acc[m][2];
+                const float u = lane == 0 ? acc[m][1] : acc[m][3];
+                const int j = (n0 >> 1) + lane;
+                if (lane < 2 && 2 * j + 1 < op.N) op.out[(size_t)m * op.ldo + j] = (g / (1.0f + expf(-g))) * u;
+            }
+        }
+    }
+}
+
+template <int M, int MB>
+__device__ void run_gemv_op(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it) {
+    float lv[1]; int li[1];
+    switch (op.mode) {
+        case kStore: gemv_consume<M, kStore, true, MB>(a, op, sh, it, lv, li); break;
+        case kSwiglu: gemv_consume<M, kSwiglu, true, MB>(a, op, sh, it, lv, li); break;
+        default: gemv_consume<M, kResid, false, MB>(a, op, sh, it, lv, li); break;
+    }
+}
+
+// Head (one row): logits + top-8.  Per-warp lists -> CTA list -> global lists -> the last CTA to
+// arrive merges them (atomic ticket; nobody waits).
+template <int MB>
+__device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int* top_out) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    float lv[1] = {__int_as_float(0xFF800000)};
+    int li[1] = {0x7FFFFFFF};
+    gemv_consume<1, kHead, true, MB>(a, op, sh, it, lv, li);
+    if (lane < 8) { sh.lists_v[warp * 8 + lane] = lv[0]; sh.lists_i[warp * 8 + lane] = li[0]; }
+    consumer_sync();
+    int* ticket = a.state + S_HEAD_TICKET;
+    float* gv = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.head_scratch) + 256);
+    int* gi = reinterpret_cast<int*>(gv + (size_t)kMaxRows * kHeadMaxCtas * 8);
+    if (warp == 0) {
+        float ov; int oi;
+        select8(sh.lists_v, sh.lists_i, kCW * 8, lane, ov, oi);
+        if (lane < 8) { gv[blockIdx.x * 8 + lane] = ov; gi[blockIdx.x * 8 + lane] = oi; }
+    }
+    __threadfence();
+    consumer_sync();
+    if (tid == 0) sh.flags[0] = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+    consumer_sync();
+    if (sh.flags[0]) {
+        __threadfence();
+        float* sv = reinterpret_cast<float*>(sh.un);
+        int* si = reinterpret_cast<int*>(sh.un) + kHeadMaxCtas * 8;
+        const int n = (int)gridDim.x * 8;
+        float tv[kHeadMaxCtas * 8 / 256];
+        int ti[kHeadMaxCtas * 8 / 256];
+#pragma unroll
+        for (int j = 0; j < kHeadMaxCtas * 8 / 256; ++j) {
+            const int c = tid + j * 256;
+            tv[j] = c < n ? __ldcg(gv + c) : 0.f;
+            ti[j] = c < n ? __ldcg(gi + c) : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < kHeadMaxCtas * 8 / 256; ++j) {
+            const int c = tid + j * 256;
+            if (c < n) { sv[c] = tv[j]; si[c] = ti[j]; }
+        }
+        consumer_sync();
+        {   // every warp pre-selects the best 8 of its slice, then warp 0 selects among the 64
+            const int per = (n + kCW - 1) / kCW;
+            const int lo_ = min(warp * per, n), hi_ = min(lo_ + per, n);
+            float ov; int oi;
+            select8(sv + lo_, si + lo_, hi_ - lo_, lane, ov, oi);
+            if (lane < 8) { sh.lists_v[warp * 8 + lane] = ov; sh.lists_i[warp * 8 + lane] = oi; }
+        }
+        consumer_sync();
+        if (warp == 0) {
+            float ov; int oi;
+            select8(sh.lists_v, sh.lists_i, kCW * 8, lane, ov, oi);
+            if (lane < 8) {
+                top_out[lane] = oi;
+                reinterpret_cast<float*>(top_out)[32 + lane] = ov;
+            }
+        }
+        if (tid == 0) *ticket = 0;
+        consumer_sync();
+    }
+}
+
+__device__ __forceinline__ float rot_lo(float x0, float x1, float2 cs) { return __fmaf_rn(x0, cs.x, -__fmul_rn(x1, cs.y)); }
+__device__ __forceinline__ float rot_hi(float x0, float x1, float2 cs) { return __fmaf_rn(x1, cs.x, __fmul_rn(x0, cs.y)); }
+
+// Sum over the 32 lanes of 32 per-lane values at once: after the call lane t holds the total of
+// v[t].  31 shuffles instead of 160; the order of additions is a fixed butterfly.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int half = 16; half >= 1; half >>= 1) {
+        const bool upper = (lane & half) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float keep = upper ? v[i + half] : v[i];
+            const float send = upper ? v[i] : v[i + half];
+            v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, half);
+        }
+    }
+    return v[0];
+}
+
+// Attention of one lane: this CTA's units.  A unit is one head and up to kUnitSplits consecutive
+// KV pages; its pages arrive through the ring (K tile + V tile per stage, plus the raw q rows and,
+// for the page that receives the new token, the raw k and v rows).
+//  - Each page is processed by ONE warp, so the pages of a unit run side by side: lane j owns dims
+//    [j*DPL, (j+1)*DPL) of the head; the scores of 32 positions are reduced across lanes together
+//    (lane t ends up owning positions t and t+32); softmax statistics by shuffles; P.V with the
+//    probabilities broadcast from their owner lanes.
+//  - A warp folds its pages (local index w, w+8) into a running (max, sum, P.V) in registers; the 8
+//    warp states are then merged through shared memory in warp order.  Up to 1024 positions of
+//    context a head is finished inside one CTA: no partial results in global memory, no tickets.
+//  - Longer contexts have R > 1 units per head; each writes one record and the last unit to
+//    register (atomic ticket, nobody waits) merges the R records in order.
+// The structure depends on the position only, never on M or on which rows share the launch.
+template <int M, int HD, int MB>
+__device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared& sh, int& it) {
+    using C = Cfg<MB>;
+    constexpr int DPL = HD / 32, HALF = HD / 2, REC = HD + 2;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x, H = a.H;
+    int* err = a.state + S_ERR;
+    const float sscale = 1.4426950408889634f / sqrtf((float)HD);
+    const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
+    const float NEG = __int_as_float(0xFF800000);
+    float* ws = reinterpret_cast<float*>(sh.un + C::kWs);          // [warp][m][REC]
+    const int d0 = lane * DPL;
+    const bool lo = d0 < HALF;
+    const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
+    float2 cs[DPL];
+#pragma unroll
+    for (int jj = 0; jj < DPL; ++jj) cs[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
+
+    for (int u = t.first_unit; u < t.units; u += G) {
+        const int h = u / t.R, r = u - h * t.R;
+        const int s_lo = r * kUnitSplits, s_hi = min(t.n_splits, s_lo + kUnitSplits);
+        float run_mx[M], run_sum[M], run_o[M][DPL];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            run_mx[m] = NEG; run_sum[m] = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = 0.f;
+        }
+        for (int s = s_lo; s < s_hi; ++s, ++it) {
+            const int slot = it % C::kStages;
+            // Every warp waits for every stage, also the ones it does not process: a warp that ran
+            // ahead would otherwise release a later use of the same ring slot too early.
+            mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
+            if ((s - s_lo) % kCW == warp) {
+                const int n_valid = min(kPageTokens, t.p - s * kPageTokens);
+                const bool tail = s == t.s_tail;
+                const uint8_t* st = sh.ring + slot * C::kStageBytes;
+                const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
+                const uint16_t* vs = ks + kPageTokens * HD;
+                const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
+                const int cnt = n_valid + (tail ? 1 : 0);      // <= 64
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    float qr[DPL], kt[DPL], vt[DPL];
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) {
+                        const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
+                        qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
+                        kt[jj] = 0.f; vt[jj] = 0.f;
+                    }
+                    if (tail) {
+                        // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
+                        const float* kr = qraw + (M + m) * HD;
+                        const float* vr = qraw + (2 * M + m) * HD;
+                        uint16_t kb[DPL], vb[DPL];
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) {
+                            const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
+                            kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
+                            vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
+                            kt[jj] = bf16_bits_to_f32(kb[jj]);
+                            vt[jj] = bf16_bits_to_f32(vb[jj]);
+                        }
+                        uint16_t *kd, *vd;
+                        if (t.slots) {
+                            kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                            vd = kd + (size_t)H * HD;
+                        } else {
+                            uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
+                            kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
+                            vd = kd + (size_t)H * kPageTokens * HD;
+                        }
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
+                    }
+                    // scores in log2 units: lane t gets positions t and t+32
+                    float sc0 = NEG, sc1 = NEG;
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {
+                        if (blk * 32 < n_valid) {
+                            float part[32];
+#pragma unroll
+                            for (int tt = 0; tt < 32; ++tt) {
+                                const int pos = blk * 32 + tt;
+                                float kf[DPL];
+                                if constexpr (DPL == 4) {
+                                    const uint2 kk = *reinterpret_cast<const uint2*>(ks + pos * HD + lane * 4);
+                                    kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
+                                } else {
+                                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + pos * HD + lane * 2);
+                                    kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
+                                }
+                                float dsum = 0.f;
+#pragma unroll
+                                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kf[jj], dsum);
+                                part[tt] = dsum;       // rows >= n_valid hold stale bytes: masked below
+                            }
+                            const float tot = transpose_reduce32(part, lane) * sscale;
+                            const bool ok = blk * 32 + lane < n_valid;
+                            if (blk == 0) sc0 = ok ? tot : NEG; else sc1 = ok ? tot : NEG;
+                        }
+                    }
+                    if (tail) {
+                        float dsum = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
+                        dsum = warp_sum(dsum) * sscale;
+                        if (n_valid < 32) { if (lane == n_valid) sc0 = dsum; }
+                        else if (lane == n_valid - 32) sc1 = dsum;
+                    }
+                    const float mx = warp_max(fmaxf(sc0, sc1));
+                    const float p0 = lane < cnt ? exp2f(sc0 - mx) : 0.f;
+                    const float p1 = lane + 32 < cnt ? exp2f(sc1 - mx) : 0.f;
+                    const float sum = warp_sum(p0 + p1);
+                    // P.V over the cached positions in ascending order, then the new token
+                    float o[DPL];
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
+                    for (int tt = 0; tt < n_valid; ++tt) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, tt < 32 ? p0 : p1, tt & 31);
+                        if constexpr (DPL == 4) {
+                            const uint2 vv = *reinterpret_cast<const uint2*>(vs + tt * HD + lane * 4);
+                            o[0] = fmaf(pw, bf16_lo(vv.x), o[0]); o[1] = fmaf(pw, bf16_hi(vv.x), o[1]);
+                            o[2] = fmaf(pw, bf16_lo(vv.y), o[2]); o[3] = fmaf(pw, bf16_hi(vv.y), o[3]);
+                        } else {
+                            const uint32_t vv = *reinterpret_cast<const uint32_t*>(vs + tt * HD + lane * 2);
+                            o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
+                        }
+                    }
+                    if (tail) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, n_valid < 32 ? p0 : p1, n_valid & 31);
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
+                    }
+                    // fold this page into the warp's running state
+                    const float nm = fmaxf(run_mx[m], mx);
+                    const float wa = exp2f(run_mx[m] - nm), wb = exp2f(mx - nm);
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = fmaf(o[jj], wb, __fmul_rn(run_o[m][jj], wa));
+                    run_sum[m] = fmaf(sum, wb, __fmul_rn(run_sum[m], wa));
+                    run_mx[m] = nm;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+        }
+        // merge the warp states (warp order) through shared memory
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float* w = ws + ((size_t)warp * M + m) * REC;
+#pragma unroll
+            for (int jj = 0; jj < DPL; ++jj) w[d0 + jj] = run_o[m][jj];
+            if (lane == 0) { w[HD] = run_mx[m]; w[HD + 1] = run_sum[m]; }
+        }
+        consumer_sync();
+        for (int idx = tid; idx < M * HD; idx += kCW * 32) {
+            const int m = idx / HD, jd = idx - m * HD;
+            float mx = ws[(size_t)m * REC + HD], num = ws[(size_t)m * REC + jd], den = ws[(size_t)m * REC + HD + 1];   // warp 0
+#pragma unroll
+            for (int w = 1; w < kCW; ++w) {
+                const float* rec = ws + ((size_t)w * M + m) * REC;
+                const float ms = rec[HD];
+                const float nm = fmaxf(mx, ms);
+                const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
+                num = fmaf(rec[jd], wb, __fmul_rn(num, wa));
+                den = fmaf(rec[HD + 1], wb, __fmul_rn(den, wa));
+                mx = nm;
+            }
+            if (t.R == 1) {
+                t.out[(size_t)m * a.Dp + h * HD + jd] = num / den;
+            } else {
+                float* rec = t.partial + (((size_t)m * H + h) * a.max_splits + r) * REC;
+                rec[jd] = num;
+                if (jd == 0) { rec[HD] = mx; rec[HD + 1] = den; }
+            }
+        }
+        consumer_sync();
+    }
+}
+
+// Contexts beyond kUnitSplits pages: after all units of the phase, one fence, then every unit
+// registers with its head's ticket; the CTA that registers a head's last unit merges that head's
+// R records in ascending order.
+template <int M, int HD, int MB>
+__device__ void attn_merge(const FusedArgs& a, const AttnDesc& t, const Shared& sh) {
+    using C = Cfg<MB>;
+    constexpr int REC = HD + 2;
+    if (t.R == 1) return;
+    const int tid = threadIdx.x;
+    const int G = gridDim.x, H = a.H;
+    float* stage = reinterpret_cast<float*>(sh.un + C::kMerge);
+    const int my_units = t.first_unit < t.units ? (t.units - 1 - t.first_unit) / G + 1 : 0;
+    for (int i0 = 0; i0 < my_units; i0 += 64) {
+        const int nb = min(64, my_units - i0);
+        if (tid < nb) {
+            const int u = t.first_unit + (i0 + tid) * G;
+            sh.flags[tid] = (atomicAdd(&t.tickets[u / t.R], 1) == t.R - 1) ? u / t.R : -1;
+        }
+        consumer_sync();
+        for (int q = 0; q < nb; ++q) {
+            const int h = sh.flags[q];
+            if (h < 0) continue;
+            __threadfence();
+            for (int m = 0; m < M; ++m) {
+                const float* part = t.partial + ((size_t)m * H + h) * a.max_splits * REC;
+                float mx = __int_as_float(0xFF800000), num = 0.f, den = 0.f;
+                for (int s0 = 0; s0 < t.R; s0 += kMergeChunk) {
+                    const int ns = min(kMergeChunk, t.R - s0);
+                    const int len = ns * REC;
+                    constexpr int LPT = (kMergeChunk * REC + 255) / 256;
+                    float tmp[LPT];
+#pragma unroll
+                    for (int u = 0; u < LPT; ++u) {
+                        const int c = tid + u * 256;
+                        tmp[u] = c < len ? __ldcg(part + (size_t)s0 * REC + c) : 0.f;
+                    }
+                    consumer_sync();
+#pragma unroll
+                    for (int u = 0; u < LPT; ++u) {
+                        const int c = tid + u * 256;
+                        if (c < len) stage[c] = tmp[u];
+                    }
+                    consumer_sync();
+                    if (tid < HD) {
+                        for (int s = 0; s < ns; ++s) {
+                            const float ms = stage[s * REC + HD];
+                            const float nm = fmaxf(mx, ms);
+                            const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
+                            num = fmaf(stage[s * REC + tid], wb, __fmul_rn(num, wa));
+                            den = fmaf(stage[s * REC + HD + 1], wb, __fmul_rn(den, wa));
+                            mx = nm;
+                        }
+                    }
+                }
+                if (tid < HD) t.out[(size_t)m * a.Dp + h * HD + tid] = num / den;
+            }
+            if (tid == 0) t.tickets[h] = 0;
+        }
+        consumer_sync();
+    }
+}
+
+template <int M, int MB>
+__device__ void run_attn(const FusedArgs& a, const AttnDesc& t, const Shared& sh, int& it) {
+    if (a.hd == 128) attn_consume<M, 128, MB>(a, t, sh, it);
+    else attn_consume<M, 64, MB>(a, t, sh, it);
+}
+
+template <int M, int MB>
+__device__ void run_attn_merge(const FusedArgs& a, const AttnDesc& t, const Shared& sh) {
+    if (a.hd == 128) attn_merge<M, 128, MB>(a, t, sh);
+    else attn_merge<M, 64, MB>(a, t, sh);
+}
+
+// verify + commit (Algorithm 2): on a match the branch's K/V of layers 1..b go to cache position
+// pos+1 and its hidden state becomes the main one.  CTA c copies layers c, c+G, ...
+__device__ void commit_copy(const FusedArgs& a, const Prog& P) {
+    if (P.mode != kPpdStep) return;
+    const int token = __ldcg(a.top_final);
+    int istar = -1;
+    for (int i = 0; i < P.k; ++i)
+        if (__ldcg(a.top_early + i) == token) istar = i;
+    if (istar < 0) return;
+    const int tid = threadIdx.x;
+    const int np = P.pos + 1;
+    const int page = __ldg(a.page_table + np / kPageTokens);
+    const int hw = a.hd / 2;
+    const size_t page_elems = (size_t)2 * a.H * kPageTokens * a.hd;
+    for (int l = blockIdx.x; l < P.b; l += gridDim.x) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(a.slots + (size_t)istar * a.slot_stride + (size_t)l * a.slot_layer_stride);
+        uint16_t* pg = a.kv + (size_t)l * a.kv_layer_elems + (size_t)page * page_elems;
+        for (int w = tid; w < 2 * a.H * hw; w += kCW * 32) {
+            const int kv = w / (a.H * hw), rem = w % (a.H * hw), h = rem / hw, j = rem % hw;
+            uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)(kv * a.H + h) * kPageTokens + (np % kPageTokens)) * a.hd);
+            dst[j] = __ldcg(src + w);
+        }
+    }
+    if (blockIdx.x == gridDim.x - 1)
+        for (int i = tid; i < a.D; i += kCW * 32) a.main.h[i] = __ldcg(a.br.h + (size_t)istar * a.Dp + i);
+}
+
+__device__ void state_update(const FusedArgs& a, const Prog& P) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    unsigned long long* base = reinterpret_cast<unsigned long long*>(a.state + S_BAR_BASE);
+    *base = *base + (unsigned long long)P.n_phases * gridDim.x;
+    if (P.mode == kPrefillToken) return;
+    const int token = __ldcg(a.top_final);
+    int istar = -1;
+    if (P.mode == kPpdStep)
+        for (int i = 0; i < P.k; ++i)
+            if (__ldcg(a.top_early + i) == token) istar = i;
+    const int step = a.state[S_STEP];
+    a.out_tokens[step] = token;
+    a.out_hit[step] = istar >= 0 ? 1 : 0;
+    const float* fv = reinterpret_cast<const float*>(a.top_final) + 32;
+    a.out_margin[step] = __ldcg(fv) - __ldcg(fv + 1);
+    a.state[S_LAST_TOKEN] = token;
+    a.state[S_LAST_HIT] = istar >= 0 ? 1 : 0;
+    a.state[S_PENDING] = token;
+    a.state[S_POS] = P.pos + 1;
+    a.state[S_STEP] = step + 1;
+    a.state[S_PREV_HIT] = istar >= 0 ? 1 : 0;
+    a.state[S_PREV_B] = P.b;
+}
+
+template <int MB>
+__global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs a) {
+    using C = Cfg<MB>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* misc = smem + C::kStages * C::kStageBytes;
+    Shared sh;
+    sh.ring = smem;
+    sh.full = reinterpret_cast<uint64_t*>(misc);
+    sh.empty = sh.full + 8;
+    sh.phase_bar = sh.full + 16;
+    sh.un = misc + C::kBarBytes;
+    sh.lists_v = reinterpret_cast<float*>(misc + C::kBarBytes + C::kUnion);
+    sh.lists_i = reinterpret_cast<int*>(sh.lists_v + kCW * kMaxRows * 8);
+    sh.flags = reinterpret_cast<int*>(misc + C::kBarBytes + C::kUnion + C::kLists);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], kCW);
+        }
+        mbar_init(sh.phase_bar, 1);
+        sh.flags[64] = 0;   // stages armed so far (written by producer W, read by producer X)
+        fence_barrier_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();                       // the program depends on the state the previous step left
+    const Prog P = build_prog(a);
+
+    if (warp >= kCW) {
+        volatile int* n_w_pub = reinterpret_cast<volatile int*>(sh.flags + 64);
+        if (tid == kCW * 32) producer_w<MB>(a, P, smem, sh.full, sh.empty, n_w_pub);
+        if (tid == (kCW + 1) * 32) producer_x<MB>(a, P, smem, sh.full, sh.phase_bar, n_w_pub);
+        return;
+    }
+
+    int* err = a.state + S_ERR;
+    unsigned long long* cnt = reinterpret_cast<unsigned long long*>(a.state + S_BAR_COUNT);
+    int it = 0;
+    PhaseDesc pd;
+    for (int ph = 0; ph < P.n_phases; ++ph) {
+        mbar_wait(sh.phase_bar, ph & 1, err, kErrPhaseWait);
+        make_phase(a, P, ph, MB, pd);
+        const bool trace = a.timeline && tid == 0 && ph < a.timeline_phases && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1);
+        unsigned long long* tl = a.timeline + ((size_t)(blockIdx.x == 0 ? 0 : 1) * a.timeline_phases + ph) * 2;
+        if (trace) tl[0] = global_timer_ns();
+        switch (pd.kind) {
+            case PH_EMBED_MAIN:
+                if (blockIdx.x == 0) {
+                    const int tok = a.mode == kPrefillToken ? __ldcg(a.token_src) : __ldcg(a.state + S_PENDING);
+                    const uint16_t* e = a.emb + (size_t)tok * a.D;
+                    for (int i = tid; i < a.D; i += kCW * 32) a.main.h[i] = bf16_bits_to_f32(e[i]);
+                }
+                break;
+            case PH_EMBED_BR:
+                if ((int)blockIdx.x < P.k) {
+                    const uint16_t* e = a.emb + (size_t)__ldcg(a.top_early + blockIdx.x) * a.D;
+                    for (int i = tid; i < a.D; i += kCW * 32) a.br.h[(size_t)blockIdx.x * a.Dp + i] = bf16_bits_to_f32(e[i]);
+                }
+                break;
+            case PH_QKV: case PH_O: case PH_GU: case PH_DOWN:
+                run_gemv_op<1, MB>(a, pd.op[0], sh, it);
+                if (MB > 0 && pd.n_ops == 2) run_gemv_op<(MB > 0 ? MB : 1), MB>(a, pd.op[1], sh, it);
+                break;
+            case PH_ATTN:
+                run_attn<1, MB>(a, pd.at[0], sh, it);
+                if (MB > 0 && pd.n_ops == 2) run_attn<(MB > 0 ? MB : 1), MB>(a, pd.at[1], sh, it);
+                __threadfence();
+                consumer_sync();
+                run_attn_merge<1, MB>(a, pd.at[0], sh);
+                if (MB > 0 && pd.n_ops == 2) run_attn_merge<(MB > 0 ? MB : 1), MB>(a, pd.at[1], sh);
+                break;
+            case PH_HEAD_EARLY:
+                run_head<MB>(a, pd.op[0], sh, it, a.top_early);
+                break;
+            case PH_HEAD_FINAL:
+                run_head<MB>(a, pd.op[0], sh, it, a.top_final);
+                break;
+            case PH_COMMIT:
+                commit_copy(a, P);
+                break;
+            default:
+                state_update(a, P);
+                break;
+        }
+        // grid barrier arrival: everything this CTA wrote in the phase is visible before the count moves
+        if (trace) tl[1] = global_timer_ns();
+        // the CTA barrier orders every consumer's writes before thread 0's fence (cumulativity)
+        consumer_sync();
+        if (tid == 0) {
+            __threadfence();
+            asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(cnt) : "memory");
+        }
+    }
+}
+
+template <int MB>
+cudaError_t launch_mb(const FusedArgs& a, cudaStream_t st, bool pdl, int n_sms) {
+    using C = Cfg<MB>;
+    static_assert(C::kStages >= 3, "ring too shallow");
+    static bool configured = false;
+    auto kern = fused_step_kernel<MB>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_sms < kHeadMaxCtas ? n_sms : kHeadMaxCtas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmem;
+    cfg.stream = st;
+    // One CTA per SM by shared-memory footprint, grid <= SM count: all CTAs are resident together,
+    // which the grid barriers need.
+    cudaLaunchAttribute attr[1];
+    int n = 0;
+    if (pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+}  // namespace
+
+cudaError_t launch_fused_step(const FusedArgs& a, int mb, cudaStream_t st, bool pdl, int n_sms) {
+    switch (mb) {
+        case 0: return launch_mb<0>(a, st, pdl, n_sms);
+        case 1: return launch_mb<1>(a, st, pdl, n_sms);
+        case 2: return launch_mb<2>(a, st, pdl, n_sms);
+        case 3: return launch_mb<3>(a, st, pdl, n_sms);
+        case 4: return launch_mb<4>(a, st, pdl, n_sms);
+        case 5: return launch_mb<5>(a, st, pdl, n_sms);
+        case 6: return launch_mb<6>(a, st, pdl, n_sms);
+        case 7: return launch_mb<7>(a, st, pdl, n_sms);
+        case 8: return launch_mb<8>(a, st, pdl, n_sms);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace ppd

@@ -37,6 +37,8 @@ cudaError_t launch_pack(const void* src, bool src_f32, int n_rows, int n_cols, u
 cudaError_t launch_convert(const void* src, bool src_f32, void* dst, bool dst_f32, size_t n, cudaStream_t st);
 cudaError_t launch_rope_table(float2* table, int n_pos, int hd, double theta, cudaStream_t st);
 cudaError_t launch_commit(const CommitArgs& a, cudaStream_t st, bool pdl);
+struct WordWrites { int n; int idx[8]; int val[8]; };   // base[idx[i]] = val[i]
+cudaError_t launch_write_words(int* base, const WordWrites& w, cudaStream_t st);
 cudaError_t launch_set_state(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step, cudaStream_t st);
 
 }  // namespace ppd

@@ -10,6 +10,7 @@
 
 #include "../../include/ppd.h"
 #include "common.cuh"
+#include "fused_step.cuh"
 #include "gemv.cuh"
 #include "misc.cuh"
 
@@ -19,6 +20,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr size_t kStagingBytes = 64ull << 20;
+constexpr int kTimelinePhases = 512;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int round_up(int v, int a) { return (v + a - 1) / a * a; }
@@ -33,7 +35,7 @@ struct Layout {
     size_t ws[2];            // main / branch workspaces
     size_t ws_h, ws_qkv, ws_attn, ws_z, ws_part, ws_tick, ws_bytes[2];   // offsets inside a workspace
     size_t logits_final, logits_early, top_final, top_early, head_scratch;
-    size_t state, prompt, out_tokens, out_hit, out_margin, staging, total;
+    size_t state, prompt, out_tokens, out_hit, out_margin, timeline, staging, total;
 };
 
 bool valid_config(const ppd_config* c) {
@@ -106,13 +108,11 @@ Layout plan(const ppd_config& c) {
     L.out_tokens = take((size_t)c.max_seq * 4);
     L.out_hit = take((size_t)c.max_seq);
     L.out_margin = take((size_t)c.max_seq * 4);
+    L.timeline = take(kTimelinePhases * 2 * 2 * 8);
     L.staging = take(kStagingBytes);
     L.total = o;
     return L;
 }
-
-// indices into the device state block (ints)
-enum { S_POS = 0, S_PENDING = 1, S_STEP = 2, S_TICKET = 3, S_LAST_TOKEN = 4, S_LAST_HIT = 5, S_ERR = 6 };
 
 struct Lane {      // one activation workspace (main: 1 row, branch: up to max_k rows)
     float *h, *qkv, *attn, *z, *partial;
@@ -137,6 +137,11 @@ struct ppd_ctx {
     cudaError_t cuda_err;
     Lane lane[2];
     int* state;
+    bool trace;                       // record per-phase timestamps of the fused kernel
+    bool fused;                       // true: one persistent kernel per step; false: per-op kernels on two streams
+    std::vector<cudaEvent_t> step_ev; // per-step timing events of the fused path (grown on demand)
+    std::vector<int32_t> h_tokens;    // staging for the bulk read-back
+    std::vector<uint8_t> h_hits;
 };
 
 namespace {
@@ -252,8 +257,30 @@ int finish_step(ppd_ctx* x, int32_t* token, uint8_t* hit) {
     return PPD_OK;
 }
 
+int enqueue_fused_step(ppd_ctx* x, int k, int l);
+int sync_state(ppd_ctx* x);
+
 // One decode step.  k = 0: conventional greedy step.  k >= 1: PPD step with early layer l.
 int decode_step(ppd_ctx* x, int k, int l, int32_t* token, uint8_t* hit) {
+    if (x->fused) {
+        int rc;
+        const bool cont = x->prev_hit && !(k > 0 && x->prev_b > l);
+        CK(cudaEventRecord(x->ev_t0, x->sm));
+        if ((rc = enqueue_fused_step(x, k, l))) return rc;
+        CK(cudaEventRecord(x->ev_t1, x->sm));
+        CK(cudaMemcpyAsync(x->h_last, x->state + S_LAST_TOKEN, 3 * sizeof(int), cudaMemcpyDeviceToHost, x->sm));
+        if ((rc = sync_state(x))) return rc;
+        *token = x->h_last[0];
+        *hit = (uint8_t)x->h_last[1];
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, x->ev_t0, x->ev_t1));
+        x->stats.steps += 1;
+        x->stats.hits += *hit;
+        if (cont) { x->stats.steps_after_hit += 1; x->stats.ms_steps_cont += ms; }
+        else x->stats.ms_steps_fresh += ms;
+        x->stats.ms_decode += ms;
+        return PPD_OK;
+    }
     const ppd_config& c = x->c;
     const Layout& L = x->L;
     const int d = c.n_layers;
@@ -302,6 +329,125 @@ int decode_step(ppd_ctx* x, int k, int l, int32_t* token, uint8_t* hit) {
     x->prev_b = b;
     x->pos += 1;
     x->pending = *token;
+    {
+        WordWrites ww{2, {S_PREV_HIT, S_PREV_B}, {x->prev_hit ? 1 : 0, b}};
+        CK(launch_write_words(x->state, ww, x->sm));
+    }
+    return PPD_OK;
+}
+
+// ---------------------------------------------------------------- fused (persistent-kernel) path
+
+void fill_fused(ppd_ctx* x, FusedArgs& f) {
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    f = FusedArgs{};
+    f.d = c.n_layers; f.D = c.d_model; f.F = c.d_ffn; f.V = c.vocab; f.H = c.n_heads; f.hd = c.head_dim;
+    f.Dp = L.Dp; f.Fp = L.Fp; f.eps = c.rms_eps;
+    f.layers = x->base + L.layers; f.layer_bytes = (long long)L.layer_bytes;
+    f.off_wqkv = (long long)L.off_wqkv; f.off_wo = (long long)L.off_wo; f.off_wgu = (long long)L.off_wgu;
+    f.off_wd = (long long)L.off_wd; f.off_g1 = (long long)L.off_g1; f.off_g2 = (long long)L.off_g2;
+    f.emb = at<uint16_t>(x, L.emb); f.g_final = at<float>(x, L.g_final); f.w_head = at<uint16_t>(x, L.w_head);
+    f.kv = at<uint16_t>(x, L.kv); f.kv_layer_elems = L.kv_layer_elems; f.page_table = at<int>(x, L.page_table);
+    f.slots = at<uint16_t>(x, L.slots); f.slot_stride = L.slot_elems; f.slot_layer_stride = L.slot_layer_elems;
+    f.rope = at<float2>(x, L.rope); f.max_splits = L.max_splits;
+    for (int w = 0; w < 2; ++w) {
+        LaneBuf& b = w == 0 ? f.main : f.br;
+        b.h = x->lane[w].h; b.qkv = x->lane[w].qkv; b.attn = x->lane[w].attn; b.z = x->lane[w].z;
+        b.partial = x->lane[w].partial; b.tickets = x->lane[w].tickets;
+    }
+    f.logits_early = at<float>(x, L.logits_early); f.logits_final = at<float>(x, L.logits_final);
+    f.top_early = at<int>(x, L.top_early); f.top_final = at<int>(x, L.top_final);
+    f.head_scratch = at<void>(x, L.head_scratch);
+    f.state = x->state;
+    f.out_tokens = at<int>(x, L.out_tokens); f.out_hit = at<uint8_t>(x, L.out_hit); f.out_margin = at<float>(x, L.out_margin);
+    f.timeline = x->trace ? at<unsigned long long>(x, L.timeline) : nullptr;
+    f.timeline_phases = kTimelinePhases;
+}
+
+// Enqueues one decode step (greedy for k = 0) as a single launch; nothing is read back.
+int enqueue_fused_step(ppd_ctx* x, int k, int l) {
+    FusedArgs f;
+    fill_fused(x, f);
+    f.mode = k > 0 ? kPpdStep : kGreedyStep;
+    f.k = k; f.l = l;
+    CK(launch_fused_step(f, k, x->sm, x->pdl, x->n_sms));
+    x->stats.kernel_launches += 1;
+    return PPD_OK;
+}
+
+int ensure_events(ppd_ctx* x, size_t n) {
+    while (x->step_ev.size() < n) {
+        cudaEvent_t e;
+        CK(cudaEventCreate(&e));
+        x->step_ev.push_back(e);
+    }
+    return PPD_OK;
+}
+
+// Reads the host mirrors (position, pending token, committed-branch state, error word) back.
+int sync_state(ppd_ctx* x) {
+    int w[16];
+    CK(cudaMemcpyAsync(w, x->state, sizeof(w), cudaMemcpyDeviceToHost, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    if (w[S_ERR] != 0) return PPD_ETIMEOUT;
+    x->pos = w[S_POS]; x->pending = w[S_PENDING]; x->prev_hit = w[S_PREV_HIT] != 0; x->prev_b = w[S_PREV_B];
+    return PPD_OK;
+}
+
+// n steps enqueued back to back (no host round trip between steps), then one read-back.
+int decode_fused(ppd_ctx* x, int k, int l, int n, int eos, int32_t* out_tokens, uint8_t* out_hit, int32_t* out_n) {
+    const Layout& L = x->L;
+    int rc;
+    const int chunk = eos >= 0 ? 1 : n;     // a stop token needs the host to look at every token
+    int done = 0;
+    x->stats.ms_decode = 0.0;
+    bool prev_hit = x->prev_hit;
+    while (done < n) {
+        const int m = n - done < chunk ? n - done : chunk;
+        WordWrites ww{1, {S_STEP}, {0}};
+        CK(launch_write_words(x->state, ww, x->sm));
+        if ((rc = ensure_events(x, (size_t)m + 1))) return rc;
+        CK(cudaEventRecord(x->step_ev[0], x->sm));
+        for (int s = 0; s < m; ++s) {
+            if ((rc = enqueue_fused_step(x, k, l))) return rc;
+            CK(cudaEventRecord(x->step_ev[s + 1], x->sm));
+        }
+        x->h_tokens.resize(m);
+        x->h_hits.resize(m);
+        CK(cudaMemcpyAsync(x->h_tokens.data(), x->base + L.out_tokens, (size_t)m * 4, cudaMemcpyDeviceToHost, x->sm));
+        CK(cudaMemcpyAsync(x->h_hits.data(), x->base + L.out_hit, (size_t)m, cudaMemcpyDeviceToHost, x->sm));
+        if ((rc = sync_state(x))) return rc;
+        bool stop = false;
+        for (int s = 0; s < m; ++s) {
+            float ms = 0.f;
+            CK(cudaEventElapsedTime(&ms, x->step_ev[s], x->step_ev[s + 1]));
+            x->stats.steps += 1;
+            x->stats.hits += x->h_hits[s];
+            if (prev_hit) { x->stats.steps_after_hit += 1; x->stats.ms_steps_cont += ms; }
+            else x->stats.ms_steps_fresh += ms;
+            x->stats.ms_decode += ms;
+            prev_hit = x->h_hits[s] != 0;
+            out_tokens[done + s] = x->h_tokens[s];
+            out_hit[done + s] = x->h_hits[s];
+            *out_n = done + s + 1;
+            if (eos >= 0 && x->h_tokens[s] == eos) stop = true;
+        }
+        done += m;
+        if (stop) break;
+    }
+    return PPD_OK;
+}
+
+int prefill_fused(ppd_ctx* x, int n_prompt) {
+    FusedArgs f;
+    fill_fused(x, f);
+    f.mode = kPrefillToken;
+    for (int t = 0; t + 1 < n_prompt; ++t) {
+        f.token_src = at<int>(x, x->L.prompt) + t;
+        f.pos_val = t;
+        CK(launch_fused_step(f, 0, x->sm, x->pdl, x->n_sms));
+    }
     return PPD_OK;
 }
 
@@ -348,6 +494,8 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     x->sb = reinterpret_cast<cudaStream_t>(stream_branch);
     x->loaded = x->prefilled = false;
     x->pdl = true;
+    x->fused = true;
+    x->trace = false;
     x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
     x->cuda_err = cudaSuccess;
     std::memset(&x->stats, 0, sizeof(x->stats));
@@ -395,6 +543,7 @@ void ppd_destroy(ppd_ctx* x) {
     cudaEventDestroy(x->ev_branch);
     cudaEventDestroy(x->ev_t0);
     cudaEventDestroy(x->ev_t1);
+    for (cudaEvent_t e : x->step_ev) cudaEventDestroy(e);
     cudaFreeHost(x->h_last);
     delete x;
 }
@@ -468,13 +617,21 @@ int ppd_prefill(ppd_ctx* x, const int32_t* prompt, int32_t n_prompt) {
     CK(cudaMemcpyAsync(x->base + L.prompt, prompt, (size_t)n_prompt * 4, cudaMemcpyHostToDevice, x->sm));
     CK(cudaStreamSynchronize(x->sm));   // the host array may be reused by the caller
     const int64_t launches = x->stats.kernel_launches;
-    for (int t = 0; t + 1 < n_prompt; ++t) {
-        CK(launch_embed(at<uint16_t>(x, L.emb), at<int>(x, L.prompt) + t, 1, x->c.d_model, x->lane[0].h, L.Dp, x->sm, x->pdl));
-        int rc = run_layers(x, 0, 1, 0, x->c.n_layers, nullptr, t, false, x->sm);
+    if (x->fused) {
+        int rc = prefill_fused(x, n_prompt);
         if (rc) return rc;
+    } else {
+        for (int t = 0; t + 1 < n_prompt; ++t) {
+            CK(launch_embed(at<uint16_t>(x, L.emb), at<int>(x, L.prompt) + t, 1, x->c.d_model, x->lane[0].h, L.Dp, x->sm, x->pdl));
+            int rc = run_layers(x, 0, 1, 0, x->c.n_layers, nullptr, t, false, x->sm);
+            if (rc) return rc;
+        }
     }
     x->stats.kernel_launches = launches;   // counted for decode steps only
-    CK(launch_set_state(x->state + S_POS, n_prompt - 1, x->state + S_PENDING, prompt[n_prompt - 1], x->state + S_STEP, 0, x->sm));
+    {
+        WordWrites ww{4, {S_POS, S_PENDING, S_STEP, S_PREV_HIT}, {n_prompt - 1, prompt[n_prompt - 1], 0, 0}};
+        CK(launch_write_words(x->state, ww, x->sm));
+    }
     CK(cudaMemcpyAsync(x->h_last, x->state + S_LAST_TOKEN, 3 * sizeof(int), cudaMemcpyDeviceToHost, x->sm));
     CK(cudaStreamSynchronize(x->sm));
     if (x->h_last[2] != 0) return PPD_ETIMEOUT;
@@ -499,6 +656,7 @@ int ppd_decode(ppd_ctx* x, int32_t k, int32_t l, int32_t n_tokens, int32_t eos, 
     *out_n = 0;
     int rc = check_decode_args(x, k, l, n_tokens);
     if (rc) return rc;
+    if (x->fused) return n_tokens > 0 ? decode_fused(x, k, l, n_tokens, eos, out_tokens, out_hit, out_n) : PPD_OK;
     x->stats.ms_decode = 0.0;
     for (int s = 0; s < n_tokens; ++s) {
         int32_t tok;
@@ -520,7 +678,11 @@ int ppd_step(ppd_ctx* x, int32_t k, int32_t l, const int32_t* in_token, int32_t*
     if (in_token) {
         if (*in_token < 0 || *in_token >= x->c.vocab) return PPD_EINVAL;
         CK(cudaMemcpyAsync(x->state + S_PENDING, in_token, 4, cudaMemcpyHostToDevice, x->sm));
-        if (*in_token != x->pending) x->prev_hit = false;
+        if (*in_token != x->pending) {      // a committed branch belongs to the old token
+            x->prev_hit = false;
+            WordWrites ww{1, {S_PREV_HIT}, {0}};
+            CK(launch_write_words(x->state, ww, x->sm));
+        }
         x->pending = *in_token;
     }
     return decode_step(x, k, l, out_token, out_hit);
@@ -530,7 +692,10 @@ int ppd_rewind(ppd_ctx* x, int32_t pos, int32_t pending_token) {
     if (!x || pos < 0 || pos >= x->c.max_seq || pending_token < 0 || pending_token >= x->c.vocab) return PPD_EINVAL;
     if (!x->loaded || !x->prefilled) return PPD_ESTATE;
     if (pos > x->pos) return PPD_EINVAL;
-    CK(launch_set_state(x->state + S_POS, pos, x->state + S_PENDING, pending_token, x->state + S_STEP, 0, x->sm));
+    {
+        WordWrites ww{4, {S_POS, S_PENDING, S_STEP, S_PREV_HIT}, {pos, pending_token, 0, 0}};
+        CK(launch_write_words(x->state, ww, x->sm));
+    }
     CK(cudaStreamSynchronize(x->sm));
     x->pos = pos;
     x->pending = pending_token;
@@ -539,6 +704,18 @@ int ppd_rewind(ppd_ctx* x, int32_t pos, int32_t pending_token) {
 }
 
 int32_t ppd_position(const ppd_ctx* x) { return x ? x->pos : -1; }
+
+int ppd_set_mode(ppd_ctx* x, int32_t fused) {
+    if (!x || (fused != 0 && fused != 1)) return PPD_EINVAL;
+    if ((fused != 0) == x->fused) return PPD_OK;
+    // a committed branch is dropped: the pending token is recomputed from layer 1 (same values)
+    WordWrites ww{1, {S_PREV_HIT}, {0}};
+    CK(launch_write_words(x->state, ww, x->sm));
+    CK(cudaStreamSynchronize(x->sm));
+    x->prev_hit = false;
+    x->fused = fused != 0;
+    return PPD_OK;
+}
 
 int ppd_get_stats(ppd_ctx* x, ppd_stats* out) {
     if (!x || !out) return PPD_EINVAL;
@@ -576,10 +753,28 @@ int ppd_debug_last(ppd_ctx* x, float* final_margin, int32_t* cand, int32_t k) {
 int ppd_debug_force_token(ppd_ctx* x, int32_t token) {
     if (!x || token < 0 || token >= x->c.vocab) return PPD_EINVAL;
     if (!x->prefilled) return PPD_ESTATE;
-    CK(launch_set_state(nullptr, 0, x->state + S_PENDING, token, nullptr, 0, x->sm));
+    {
+        const bool keep = token == x->pending && x->prev_hit;   // a committed branch belongs to the old token
+        WordWrites ww{2, {S_PENDING, S_PREV_HIT}, {token, keep ? 1 : 0}};
+        CK(launch_write_words(x->state, ww, x->sm));
+    }
     CK(cudaStreamSynchronize(x->sm));
-    if (token != x->pending) x->prev_hit = false;   // a committed branch belongs to the old token
+    if (token != x->pending) x->prev_hit = false;
     x->pending = token;
+    return PPD_OK;
+}
+
+int ppd_debug_phase_times(ppd_ctx* x, int32_t enable, uint64_t* out, int32_t n_phases) {
+    if (!x || n_phases < 0 || n_phases > kTimelinePhases) return PPD_EINVAL;
+    if (out && n_phases > 0) {
+        // layout: [cta 0 | last cta][phase][start, end]; copy the first n_phases of each
+        for (int c = 0; c < 2; ++c)
+            CK(cudaMemcpyAsync(out + (size_t)c * n_phases * 2, x->base + x->L.timeline + (size_t)c * kTimelinePhases * 16,
+                               (size_t)n_phases * 16, cudaMemcpyDeviceToHost, x->sm));
+        CK(cudaStreamSynchronize(x->sm));
+    }
+    if (enable) CK(cudaMemsetAsync(x->base + x->L.timeline, 0, kTimelinePhases * 32, x->sm));
+    x->trace = enable != 0;
     return PPD_OK;
 }
 

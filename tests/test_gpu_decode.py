@@ -33,10 +33,11 @@ def gpu_stream(ctx, k, l, n, forced=None):
     return np.array(toks), np.array(hits), np.array(fl), (np.array(el) if el else None), (np.array(cands) if cands else None)
 
 
-def check_against_oracle(shape, blob, prompt, n, k, l, ctx=None, max_k=8):
+def check_against_oracle(shape, blob, prompt, n, k, l, ctx=None, max_k=8, fused=True):
     own = ctx is None
     if own:
         ctx = ppd.Context(shape, max_seq=len(prompt) + n + 2, max_k=max_k)
+        ctx.set_mode(fused)
         ctx.load_weights(blob)
     ctx.prefill(prompt)
     o = Oracle(shape, blob, max_seq=len(prompt) + n + 2, max_k=max_k)
@@ -61,9 +62,11 @@ def check_against_oracle(shape, blob, prompt, n, k, l, ctx=None, max_k=8):
     return dict(max_err=float(np.abs(fl - ref["final_logits"]).max()), below_margin=int((~safe).sum()))
 
 
-@pytest.fixture(scope="module")
-def tiny_ctx(tiny_shape, tiny_blob):
+@pytest.fixture(scope="module", params=[True, False], ids=["fused", "per-op"])
+def tiny_ctx(request, tiny_shape, tiny_blob):
+    """One context per execution mode: the persistent step kernel, and per-op kernels on two streams."""
     ctx = ppd.Context(tiny_shape, max_seq=400, max_k=8)
+    ctx.set_mode(request.param)
     ctx.load_weights(tiny_blob)
     yield ctx
     ctx.close()
@@ -117,7 +120,7 @@ def test_both_hit_and_miss_paths_run(tiny_ctx, tiny_prompt):
     st = tiny_ctx.stats()
     assert 0 < hit.sum() < 32
     assert st.steps == 32 and st.hits == hit.sum() and st.steps_after_hit == hit[:-1].sum()
-    assert st.kernel_launches > 32 * 20
+    assert st.kernel_launches >= 32        # one launch per step (fused) or one per operation
 
 
 def test_greedy_step_api_and_mixed_continuation(tiny_ctx, tiny_prompt):
@@ -195,12 +198,30 @@ def test_error_codes(tiny_shape, tiny_blob, tiny_prompt):
     ctx.close()
 
 
-def test_7b_shaped_two_layers_against_oracle():
+@pytest.mark.parametrize("fused", [True, False], ids=["fused", "per-op"])
+def test_7b_shaped_two_layers_against_oracle(fused):
     # full-width shapes of the 7B workload (D 4096, F 11008 = 43 column chunks, V 32000, hd 128), 2 layers
     shape = ppd_inputs.LLAMA_7B.with_layers(2)
     blob = ppd_inputs.gen_weights(shape, seed=0)
     prompt = ppd_inputs.gen_prompt(shape.vocab, 6, seed=1)
-    check_against_oracle(shape, blob, prompt, 5, 3, 1, max_k=3)
+    check_against_oracle(shape, blob, prompt, 5, 3, 1, max_k=3, fused=fused)
+
+
+def test_modes_agree_and_can_be_switched(tiny_shape, tiny_blob, tiny_prompt):
+    ctx = ppd.Context(tiny_shape, max_seq=96, max_k=5)
+    ctx.load_weights(tiny_blob)
+    ctx.prefill(tiny_prompt)
+    ref, _ = ctx.decode(0, 0, 30)
+    ctx.set_mode(False)
+    ctx.prefill(tiny_prompt)
+    a, _ = ctx.decode(3, 2, 10)
+    ctx.set_mode(True)                 # mid-stream switch: a committed branch is dropped, tokens continue
+    b, _ = ctx.decode(5, 3, 10)
+    ctx.set_mode(False)
+    c, _ = ctx.decode(0, 0, 10)
+    # the two modes round differently, so their streams may part only at a near-tie; on this seed they agree
+    assert (np.concatenate([a, b, c]) == ref).all()
+    ctx.close()
 
 
 def test_7b_full_depth_sampled_steps_against_oracle():
@@ -213,6 +234,9 @@ def test_7b_full_depth_sampled_steps_against_oracle():
     ctx = ppd.Context(shape, max_seq=1024, max_k=3)
     ctx.load_weights(blob)
     r = check_against_oracle(shape, blob, prompt, n, 3, 16, ctx=ctx, max_k=3)
+    ctx.set_mode(False)
+    check_against_oracle(shape, blob, prompt, n, 3, 16, ctx=ctx, max_k=3)
+    ctx.set_mode(True)
     # invariants that hold at any size: PPD == greedy bit for bit over a longer run
     ctx.prefill(prompt)
     g, _, gfl, _, _ = gpu_stream(ctx, 0, 0, 24)
