@@ -213,8 +213,8 @@ int ppd_op_head_topk_static(const void* w_packed, int32_t vocab, int32_t K, cons
 /* Decode attention for M query rows that share a cached prefix (Section 3: every process is fed
  * the same history x_<=t plus its own candidate).
  *   qkv: device float32 [M][3*D] un-rotated q|k|v of the M new tokens, all at position n_prefix.
- *   kv_pages: device bf16, one layer's pages; a page holds K as [H][64][hd] followed by V
- *   transposed as [H][hd][64]; page_table: device int32, logical page -> physical page.
+ *   kv_pages: device bf16, one layer's pages; page p holds [2 (K,V)][H][64][hd]; page_table:
+ *   device int32, logical page -> physical page.
  *   Row m attends to cached positions 0..n_prefix-1 and to its own new K/V.  The rotated,
  *   bf16-rounded K/V of row m is written to branch_slots + m*2*D (device bf16 [M][2][H][hd]) or,
  *   when branch_slots is NULL, into the cache at position n_prefix (main pass; M = 1).

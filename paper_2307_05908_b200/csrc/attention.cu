@@ -99,13 +99,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
                 kd = a.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
                 vd = kd + (size_t)H * HD;
             } else {
-                // cache page: K [H][64][hd], then V transposed [H][hd][64]
                 uint16_t* pg = a.kv_layer + (size_t)a.page_table[s_tail] * page_elems;
                 kd = pg + ((size_t)h * kPageTokens + (p % kPageTokens)) * HD;
-                uint16_t* vt = pg + (size_t)H * kPageTokens * HD + (size_t)h * HD * kPageTokens + (p % kPageTokens);
-                kd[i] = k0; kd[i + HALF] = k1;
-                vt[(size_t)i * kPageTokens] = v0; vt[(size_t)(i + HALF) * kPageTokens] = v1;
-                continue;
+                vd = kd + (size_t)H * kPageTokens * HD;
             }
             kd[i] = k0; kd[i + HALF] = k1;
             vd[i] = v0; vd[i + HALF] = v1;
@@ -176,22 +172,15 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
             if (lane == 0) { stat[2 * m] = mx; stat[2 * m + 1] = sum; }
         }
         __syncthreads();
-        // P.V with the transposed V tile [hd][64]: a warp takes one dim at a time, lane t the
-        // positions t and t+32; fixed shuffle tree over the lanes
-        for (int dim = warp; dim < HD; dim += kAttnWarps) {
-            const float v0 = lane < n_valid ? bf16_bits_to_f32(vs[dim * kPageTokens + lane]) : 0.f;
-            const float v1 = lane + 32 < n_valid ? bf16_bits_to_f32(vs[dim * kPageTokens + lane + 32]) : 0.f;
+        if (tid < HD) {
 #pragma unroll
             for (int m = 0; m < M; ++m) {
-                const float p0 = lane < n_valid ? sc[m * 68 + lane] : 0.f;
-                const float p1 = lane + 32 < n_valid ? sc[m * 68 + lane + 32] : 0.f;
-                float o = warp_sum(fmaf(p1, v1, __fmul_rn(p0, v0)));
-                if (tail) o = fmaf(sc[m * 68 + n_valid], bf16_bits_to_f32(vtail[m * HD + dim]), o);
-                if (lane == 0) {
-                    float* part = a.partial + (((size_t)m * H + h) * a.max_splits + s) * (HD + 2);
-                    part[dim] = o;
-                    if (dim == 0) { part[HD] = stat[2 * m]; part[HD + 1] = stat[2 * m + 1]; }
-                }
+                float o = 0.f;
+                for (int t = 0; t < n_valid; ++t) o = fmaf(sc[m * 68 + t], bf16_bits_to_f32(vs[t * HD + tid]), o);
+                if (tail) o = fmaf(sc[m * 68 + n_valid], bf16_bits_to_f32(vtail[m * HD + tid]), o);
+                float* part = a.partial + (((size_t)m * H + h) * a.max_splits + s) * (HD + 2);
+                part[tid] = o;
+                if (tid == 0) { part[HD] = stat[2 * m]; part[HD + 1] = stat[2 * m + 1]; }
             }
         }
         __syncthreads();

@@ -48,9 +48,7 @@ struct Cfg {
     // after the ring: barriers | union {attention warp states + merge staging, head merge staging} | head lists | flags
     static constexpr int kBarBytes = 256;
     static constexpr int kWs = 0;                                        // per-warp attention states [8 warps][MR][130] f32
-    static constexpr int kQ = kWs + kCW * MR * 130 * 4;                  // q_hi, q_lo [8][128] bf16
-    static constexpr int kNew = kQ + 2 * 8 * 128 * 2;                    // new k, v [8][128] f32
-    static constexpr int kMerge = kNew + 2 * 8 * 128 * 4;                // [kMergeChunk][130] f32
+    static constexpr int kMerge = kWs + kCW * MR * 130 * 4;              // [kMergeChunk][130] f32
     static constexpr int kUnionAttn = kMerge + kMergeChunk * 130 * 4;
     static constexpr int kUnionHead = kHeadMaxCtas * 8 * 8;              // staged candidate lists
     static constexpr int kUnion = ((kUnionAttn > kUnionHead ? kUnionAttn : kUnionHead) + 255) / 256 * 256;
@@ -235,7 +233,6 @@ struct Item {
     int rg, c0, nt;      // matrix stage
     int h, s, n_valid;   // attention stage
     bool tail;
-    bool carry_new;      // first page of the unit that receives the new token: carries its raw k, v rows
     bool kv_late;        // the K/V tile holds a position written earlier in this launch: no prefetch
 };
 
@@ -265,7 +262,6 @@ __device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P,
                         it.s = sp;
                         it.n_valid = min(kPageTokens, t.p - sp * kPageTokens);
                         it.tail = sp == t.s_tail;
-                        it.carry_new = sp == s_lo && t.s_tail >= s_lo && t.s_tail < s_hi;
                         // a branch row's prefix ends with the position the main pass wrote in this launch
                         it.kv_late = ln == 1 && sp == P.pos / kPageTokens;
                         f(pd, it);
@@ -292,7 +288,7 @@ __device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P,
 __device__ __forceinline__ uint32_t item_bytes(const FusedArgs& a, const PhaseDesc& pd, const Item& it) {
     if (it.kind == PH_ATTN) {
         const AttnDesc& t = pd.at[it.lane];
-        return (it.n_valid > 0 ? 2u * kPageTokens * a.hd * 2 : 0u) + (uint32_t)t.M * a.hd * 4 * (it.carry_new ? 3 : 1);
+        return (it.n_valid > 0 ? 2u * kPageTokens * a.hd * 2 : 0u) + (uint32_t)t.M * a.hd * 4 * (it.tail ? 3 : 1);
     }
     const OpDesc& o = pd.op[it.lane];
     return (uint32_t)it.nt * kTileBytes + (uint32_t)o.M * it.nt * kTileCols * 4 + (o.gain ? (uint32_t)it.nt * kTileCols * 4 : 0u);
@@ -325,7 +321,7 @@ __device__ __forceinline__ void issue_late(const FusedArgs& a, const PhaseDesc& 
         const AttnDesc& t = pd.at[it.lane];
         if (it.n_valid > 0 && it.kv_late) issue_kv(a, t, it, st, full);
         const uint32_t row = a.hd * 4;
-        const int parts = it.carry_new ? 3 : 1;   // q; the unit's first page also brings the new k and v rows
+        const int parts = it.tail ? 3 : 1;   // q, and for the tail split the new k and v rows
         for (int part = 0; part < parts; ++part)
             for (int m = 0; m < t.M; ++m)
                 bulk_g2s(st + C::kXOff + (part * t.M + m) * row, t.qkv + (size_t)m * 3 * a.D + part * a.D + it.h * a.hd, row, full);
@@ -650,124 +646,63 @@ __device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh,
 __device__ __forceinline__ float rot_lo(float x0, float x1, float2 cs) { return __fmaf_rn(x0, cs.x, -__fmul_rn(x1, cs.y)); }
 __device__ __forceinline__ float rot_hi(float x0, float x1, float2 cs) { return __fmaf_rn(x1, cs.x, __fmul_rn(x0, cs.y)); }
 
-// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col).  Rows 8..15 of A are always zero here
-// (at most 8 query rows), so a1 = a3 = 0 and only c0, c1 (rows 0..7) carry results.
-__device__ __forceinline__ void mma_bf16_rows8(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-    float c2 = 0.f, c3 = 0.f;
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
-        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+// Sum over the 32 lanes of 32 per-lane values at once: after the call lane t holds the total of
+// v[t].  31 shuffles instead of 160; the order of additions is a fixed butterfly.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int half = 16; half >= 1; half >>= 1) {
+        const bool upper = (lane & half) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float keep = upper ? v[i + half] : v[i];
+            const float send = upper ? v[i] : v[i + half];
+            v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, half);
+        }
+    }
+    return v[0];
 }
-
-// x = hi + lo with hi = bf16(x) and lo = bf16(x - hi): two bf16 MMAs then carry ~16 mantissa bits.
-__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
-    hi = f32_to_bf16_bits(x);
-    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi));
-}
-__device__ __forceinline__ uint32_t pack_u16(uint16_t a, uint16_t b) { return (uint32_t)a | ((uint32_t)b << 16); }
 
 // Attention of one lane: this CTA's units.  A unit is one head and up to kUnitSplits consecutive
-// KV pages; its pages arrive through the ring (K tile [64][hd] + transposed V tile [hd][64] per
-// stage, plus the raw q rows and, for the page that receives the new token, the raw k and v rows).
-//
-//  - Each page is processed by ONE warp with narrow tensor-core MMAs (m16n8k16, bf16 inputs, fp32
-//    accumulation): the <= 8 query rows are the rows of A, S = Q.K^T over the page, softmax
-//    statistics per row, O += P.V.  q and the probabilities are split into bf16 hi + lo parts so
-//    that the products keep ~16 mantissa bits; K and V are bf16 already.  The rows of an MMA are
-//    independent, so a row's result does not depend on how many rows share the launch.
-//  - Index mapping: thread (g = lane/4, c = lane%4) owns query row g.  In an MMA the k index and
-//    the n index are just labels, so they are permuted such that every operand register comes
-//    from a 16-byte contiguous shared-memory load: column n of score tile j is position
-//    (j/4)*32 + (n/2)*8 + (j%4)*2 + n%2, which makes thread c own the 8 consecutive positions
-//    b*32 + c*8 .. +7 of each 32-position block -- exactly one 16-byte chunk of a V^T row.
-//  - A warp folds its pages (local index w, w+8) into a running (max, sum, O) in registers; the 8
-//    warp states are merged through shared memory in warp order.  Up to 1024 positions of context
-//    a head is finished inside one CTA: no partial results in global memory, no tickets.
+// KV pages; its pages arrive through the ring (K tile + V tile per stage, plus the raw q rows and,
+// for the page that receives the new token, the raw k and v rows).
+//  - Each page is processed by ONE warp, so the pages of a unit run side by side: lane j owns dims
+//    [j*DPL, (j+1)*DPL) of the head; the scores of 32 positions are reduced across lanes together
+//    (lane t ends up owning positions t and t+32); softmax statistics by shuffles; P.V with the
+//    probabilities broadcast from their owner lanes.
+//  - A warp folds its pages (local index w, w+8) into a running (max, sum, P.V) in registers; the 8
+//    warp states are then merged through shared memory in warp order.  Up to 1024 positions of
+//    context a head is finished inside one CTA: no partial results in global memory, no tickets.
 //  - Longer contexts have R > 1 units per head; each writes one record and the last unit to
 //    register (atomic ticket, nobody waits) merges the R records in order.
 // The structure depends on the position only, never on M or on which rows share the launch.
 template <int M, int HD, int MB>
 __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared& sh, int& it) {
     using C = Cfg<MB>;
-    constexpr int HALF = HD / 2, REC = HD + 2;
-    constexpr int NB = HD / 32;          // 32-dim blocks
-    constexpr int NT = HD / 8;           // output n-tiles (8 dims each)
+    constexpr int DPL = HD / 32, HALF = HD / 2, REC = HD + 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, c = lane & 3;
     const int G = gridDim.x, H = a.H;
     int* err = a.state + S_ERR;
     const float sscale = 1.4426950408889634f / sqrtf((float)HD);
     const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
     const float NEG = __int_as_float(0xFF800000);
-    float* ws = reinterpret_cast<float*>(sh.un + C::kWs);                       // [warp][m][REC]
-    uint16_t* q_hi = reinterpret_cast<uint16_t*>(sh.un + C::kQ);               // [8][HD] bf16, rows >= M zero
-    uint16_t* q_lo = q_hi + 8 * HD;
-    float* k_new = reinterpret_cast<float*>(sh.un + C::kNew);                  // [8][HD] rotated, rounded new keys
-    float* v_new = k_new + 8 * HD;                                             // [8][HD] rounded new values
+    float* ws = reinterpret_cast<float*>(sh.un + C::kWs);          // [warp][m][REC]
+    const int d0 = lane * DPL;
+    const bool lo = d0 < HALF;
+    const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
+    float2 cs[DPL];
+#pragma unroll
+    for (int jj = 0; jj < DPL; ++jj) cs[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
 
     for (int u = t.first_unit; u < t.units; u += G) {
         const int h = u / t.R, r = u - h * t.R;
         const int s_lo = r * kUnitSplits, s_hi = min(t.n_splits, s_lo + kUnitSplits);
-        const bool unit_has_tail = t.s_tail >= s_lo && t.s_tail < s_hi;
-        // ---- unit prologue (all warps): rotated queries from the first stage's q rows; new K/V
-        {
-            const int slot = it % C::kStages;
-            mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
-            const float* qraw = reinterpret_cast<const float*>(sh.ring + slot * C::kStageBytes + C::kXOff);
-            for (int idx = tid; idx < 8 * HALF; idx += kCW * 32) {
-                const int m = idx / HALF, i = idx - m * HALF;
-                uint16_t h0 = 0, l0 = 0, h1 = 0, l1 = 0;
-                if (m < M) {
-                    const float2 cs = __ldg(a.rope + (size_t)t.p * HALF + i);
-                    const float x0 = qraw[m * HD + i], x1 = qraw[m * HD + i + HALF];
-                    split_bf16(rot_lo(x0, x1, cs), h0, l0);
-                    split_bf16(rot_hi(x0, x1, cs), h1, l1);
-                }
-                q_hi[m * HD + i] = h0; q_lo[m * HD + i] = l0;
-                q_hi[m * HD + i + HALF] = h1; q_lo[m * HD + i + HALF] = l1;
-            }
-        }
-        if (unit_has_tail) {
-            // the unit's first stage also carries the raw k and v rows of the new token(s)
-            const float* qraw = reinterpret_cast<const float*>(sh.ring + (it % C::kStages) * C::kStageBytes + C::kXOff);
-            for (int idx = tid; idx < M * HALF; idx += kCW * 32) {
-                const int m = idx / HALF, i = idx - m * HALF;
-                const float2 cs = __ldg(a.rope + (size_t)t.p * HALF + i);
-                const float* kr = qraw + (M + m) * HD;
-                const float* vr = qraw + (2 * M + m) * HD;
-                const uint16_t k0 = f32_to_bf16_bits(rot_lo(kr[i], kr[i + HALF], cs));
-                const uint16_t k1 = f32_to_bf16_bits(rot_hi(kr[i], kr[i + HALF], cs));
-                const uint16_t v0 = f32_to_bf16_bits(vr[i]);
-                const uint16_t v1 = f32_to_bf16_bits(vr[i + HALF]);
-                k_new[m * HD + i] = bf16_bits_to_f32(k0); k_new[m * HD + i + HALF] = bf16_bits_to_f32(k1);
-                v_new[m * HD + i] = bf16_bits_to_f32(v0); v_new[m * HD + i + HALF] = bf16_bits_to_f32(v1);
-                if (t.slots) {       // branch slot: [K | V][H][hd]
-                    uint16_t* kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
-                    uint16_t* vd = kd + (size_t)H * HD;
-                    kd[i] = k0; kd[i + HALF] = k1; vd[i] = v0; vd[i + HALF] = v1;
-                } else {             // cache page: K [H][64][hd], then V transposed [H][hd][64]
-                    uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
-                    uint16_t* kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
-                    uint16_t* vd = pg + (size_t)H * kPageTokens * HD + (size_t)h * HD * kPageTokens + (t.p % kPageTokens);
-                    kd[i] = k0; kd[i + HALF] = k1;
-                    vd[(size_t)i * kPageTokens] = v0; vd[(size_t)(i + HALF) * kPageTokens] = v1;
-                }
-            }
-        }
-        consumer_sync();
-        // ---- this warp's query fragments: per 32-dim block the 16-byte chunk of row g at dims blk*32 + c*8
-        uint4 qh[NB], ql[NB];
+        float run_mx[M], run_sum[M], run_o[M][DPL];
 #pragma unroll
-        for (int blk = 0; blk < NB; ++blk) {
-            qh[blk] = *reinterpret_cast<const uint4*>(q_hi + g * HD + blk * 32 + c * 8);
-            ql[blk] = *reinterpret_cast<const uint4*>(q_lo + g * HD + blk * 32 + c * 8);
-        }
-        float run_mx = NEG, run_sum = 0.f;
-        float o[NT][2];
+        for (int m = 0; m < M; ++m) {
+            run_mx[m] = NEG; run_sum[m] = 0.f;
 #pragma unroll
-        for (int n = 0; n < NT; ++n) { o[n][0] = 0.f; o[n][1] = 0.f; }
-
+            for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = 0.f;
+        }
         for (int s = s_lo; s < s_hi; ++s, ++it) {
             const int slot = it % C::kStages;
             // Every warp waits for every stage, also the ones it does not process: a warp that ran
@@ -777,119 +712,122 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                 const int n_valid = min(kPageTokens, t.p - s * kPageTokens);
                 const bool tail = s == t.s_tail;
                 const uint8_t* st = sh.ring + slot * C::kStageBytes;
-                const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);            // [64][HD]
-                const uint16_t* vts = ks + kPageTokens * HD;                             // [HD][64]
-                // ---- scores S[row g][position], log2 units.  sc[j][e]: tile j, column c*2+e
-                float sc[8][2];
+                const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
+                const uint16_t* vs = ks + kPageTokens * HD;
+                const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
+                const int cnt = n_valid + (tail ? 1 : 0);      // <= 64
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    sc[j][0] = 0.f; sc[j][1] = 0.f;
-                    // B operand column n = g is position (j/4)*32 + (g/2)*8 + (j%4)*2 + g%2
-                    const int pos = (j >> 2) * 32 + (g >> 1) * 8 + (j & 3) * 2 + (g & 1);
+                for (int m = 0; m < M; ++m) {
+                    float qr[DPL], kt[DPL], vt[DPL];
 #pragma unroll
-                    for (int blk = 0; blk < NB; ++blk) {
-                        const uint4 kk = *reinterpret_cast<const uint4*>(ks + pos * HD + blk * 32 + c * 8);
-                        mma_bf16_rows8(sc[j][0], sc[j][1], qh[blk].x, qh[blk].y, kk.x, kk.y);
-                        mma_bf16_rows8(sc[j][0], sc[j][1], qh[blk].z, qh[blk].w, kk.z, kk.w);
-                        mma_bf16_rows8(sc[j][0], sc[j][1], ql[blk].x, ql[blk].y, kk.x, kk.y);
-                        mma_bf16_rows8(sc[j][0], sc[j][1], ql[blk].z, ql[blk].w, kk.z, kk.w);
+                    for (int jj = 0; jj < DPL; ++jj) {
+                        const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
+                        qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
+                        kt[jj] = 0.f; vt[jj] = 0.f;
                     }
-                }
-                // this thread's columns are positions (j/4)*32 + c*8 + (j%4)*2 + e
-                float mx = NEG;
+                    if (tail) {
+                        // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
+                        const float* kr = qraw + (M + m) * HD;
+                        const float* vr = qraw + (2 * M + m) * HD;
+                        uint16_t kb[DPL], vb[DPL];
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int pos = (j >> 2) * 32 + c * 8 + (j & 3) * 2 + e;
-                        sc[j][e] = pos < n_valid ? sc[j][e] * sscale : NEG;
-                        mx = fmaxf(mx, sc[j][e]);
-                    }
-                float s_new = NEG;
-                if (tail) {      // the new token's own key: plain dot product, row g
-                    float d = 0.f;
-                    if (g < M) {
-#pragma unroll
-                        for (int blk = 0; blk < NB; ++blk) {
-                            const uint32_t hw[4] = {qh[blk].x, qh[blk].y, qh[blk].z, qh[blk].w};
-                            const uint32_t lw[4] = {ql[blk].x, ql[blk].y, ql[blk].z, ql[blk].w};
-#pragma unroll
-                            for (int w2 = 0; w2 < 4; ++w2) {
-                                const float* kn = k_new + g * HD + blk * 32 + c * 8 + w2 * 2;
-                                d = fmaf(bf16_lo(hw[w2]) + bf16_lo(lw[w2]), kn[0], d);
-                                d = fmaf(bf16_hi(hw[w2]) + bf16_hi(lw[w2]), kn[1], d);
-                            }
+                        for (int jj = 0; jj < DPL; ++jj) {
+                            const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
+                            kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
+                            vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
+                            kt[jj] = bf16_bits_to_f32(kb[jj]);
+                            vt[jj] = bf16_bits_to_f32(vb[jj]);
                         }
+                        uint16_t *kd, *vd;
+                        if (t.slots) {
+                            kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                            vd = kd + (size_t)H * HD;
+                        } else {
+                            uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
+                            kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
+                            vd = kd + (size_t)H * kPageTokens * HD;
+                        }
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
                     }
-                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
-                    s_new = d * sscale;
-                    mx = fmaxf(mx, s_new);
-                }
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-                // probabilities, split into bf16 hi + lo, packed as A operands of the P.V products
-                float sum = 0.f;
-                uint32_t ph[8], pl[8];
+                    // scores in log2 units: lane t gets positions t and t+32
+                    float sc0 = NEG, sc1 = NEG;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float p0 = exp2f(sc[j][0] - mx), p1 = exp2f(sc[j][1] - mx);   // exp2(-inf) = 0 for masked
-                    sum += p0 + p1;
-                    uint16_t h0, l0, h1, l1;
-                    split_bf16(p0, h0, l0);
-                    split_bf16(p1, h1, l1);
-                    ph[j] = pack_u16(h0, h1);
-                    pl[j] = pack_u16(l0, l1);
-                }
-                const float p_new = tail ? exp2f(s_new - mx) : 0.f;
-                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-                if (tail) sum += p_new;
-                // ---- rescale the running state to the new maximum, then O += P.V
-                const float nm = fmaxf(run_mx, mx);
-                const float wa = exp2f(run_mx - nm), wb = exp2f(mx - nm);
-                run_sum = fmaf(sum, wb, __fmul_rn(run_sum, wa));
-                run_mx = nm;
+                    for (int blk = 0; blk < 2; ++blk) {
+                        if (blk * 32 < n_valid) {
+                            float part[32];
 #pragma unroll
-                for (int n = 0; n < NT; ++n) {
-                    float c0 = 0.f, c1 = 0.f;
-#pragma unroll
-                    for (int b = 0; b < 2; ++b) {
-                        if (b * 32 < n_valid) {
-                            // V^T row (dim n*8 + g), positions b*32 + c*8 .. +7
-                            uint4 vv = *reinterpret_cast<const uint4*>(vts + (n * 8 + g) * kPageTokens + b * 32 + c * 8);
-                            if (b * 32 + c * 8 + 8 > n_valid) {     // ragged page: never multiply stale bytes
-                                uint32_t* w4 = reinterpret_cast<uint32_t*>(&vv);
-#pragma unroll
-                                for (int w2 = 0; w2 < 4; ++w2) {
-                                    const int p0i = b * 32 + c * 8 + w2 * 2;
-                                    if (p0i >= n_valid) w4[w2] = 0u;
-                                    else if (p0i + 1 >= n_valid) w4[w2] &= 0xFFFFu;
+                            for (int tt = 0; tt < 32; ++tt) {
+                                const int pos = blk * 32 + tt;
+                                float kf[DPL];
+                                if constexpr (DPL == 4) {
+                                    const uint2 kk = *reinterpret_cast<const uint2*>(ks + pos * HD + lane * 4);
+                                    kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
+                                } else {
+                                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + pos * HD + lane * 2);
+                                    kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
                                 }
+                                float dsum = 0.f;
+#pragma unroll
+                                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kf[jj], dsum);
+                                part[tt] = dsum;       // rows >= n_valid hold stale bytes: masked below
                             }
-                            mma_bf16_rows8(c0, c1, ph[b * 4 + 0], ph[b * 4 + 1], vv.x, vv.y);
-                            mma_bf16_rows8(c0, c1, ph[b * 4 + 2], ph[b * 4 + 3], vv.z, vv.w);
-                            mma_bf16_rows8(c0, c1, pl[b * 4 + 0], pl[b * 4 + 1], vv.x, vv.y);
-                            mma_bf16_rows8(c0, c1, pl[b * 4 + 2], pl[b * 4 + 3], vv.z, vv.w);
+                            const float tot = transpose_reduce32(part, lane) * sscale;
+                            const bool ok = blk * 32 + lane < n_valid;
+                            if (blk == 0) sc0 = ok ? tot : NEG; else sc1 = ok ? tot : NEG;
                         }
                     }
-                    if (tail && g < M) {
-                        c0 = fmaf(p_new, v_new[g * HD + n * 8 + c * 2], c0);
-                        c1 = fmaf(p_new, v_new[g * HD + n * 8 + c * 2 + 1], c1);
+                    if (tail) {
+                        float dsum = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
+                        dsum = warp_sum(dsum) * sscale;
+                        if (n_valid < 32) { if (lane == n_valid) sc0 = dsum; }
+                        else if (lane == n_valid - 32) sc1 = dsum;
                     }
-                    o[n][0] = fmaf(c0, wb, __fmul_rn(o[n][0], wa));
-                    o[n][1] = fmaf(c1, wb, __fmul_rn(o[n][1], wa));
+                    const float mx = warp_max(fmaxf(sc0, sc1));
+                    const float p0 = lane < cnt ? exp2f(sc0 - mx) : 0.f;
+                    const float p1 = lane + 32 < cnt ? exp2f(sc1 - mx) : 0.f;
+                    const float sum = warp_sum(p0 + p1);
+                    // P.V over the cached positions in ascending order, then the new token
+                    float o[DPL];
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
+                    for (int tt = 0; tt < n_valid; ++tt) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, tt < 32 ? p0 : p1, tt & 31);
+                        if constexpr (DPL == 4) {
+                            const uint2 vv = *reinterpret_cast<const uint2*>(vs + tt * HD + lane * 4);
+                            o[0] = fmaf(pw, bf16_lo(vv.x), o[0]); o[1] = fmaf(pw, bf16_hi(vv.x), o[1]);
+                            o[2] = fmaf(pw, bf16_lo(vv.y), o[2]); o[3] = fmaf(pw, bf16_hi(vv.y), o[3]);
+                        } else {
+                            const uint32_t vv = *reinterpret_cast<const uint32_t*>(vs + tt * HD + lane * 2);
+                            o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
+                        }
+                    }
+                    if (tail) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, n_valid < 32 ? p0 : p1, n_valid & 31);
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
+                    }
+                    // fold this page into the warp's running state
+                    const float nm = fmaxf(run_mx[m], mx);
+                    const float wa = exp2f(run_mx[m] - nm), wb = exp2f(mx - nm);
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = fmaf(o[jj], wb, __fmul_rn(run_o[m][jj], wa));
+                    run_sum[m] = fmaf(sum, wb, __fmul_rn(run_sum[m], wa));
+                    run_mx[m] = nm;
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
         }
-        // ---- merge the warp states (warp order) through shared memory
-        if (g < M) {
-            float* w = ws + ((size_t)warp * M + g) * REC;
+        // merge the warp states (warp order) through shared memory
 #pragma unroll
-            for (int n = 0; n < NT; ++n) { w[n * 8 + c * 2] = o[n][0]; w[n * 8 + c * 2 + 1] = o[n][1]; }
-            if (c == 0) { w[HD] = run_mx; w[HD + 1] = run_sum; }
+        for (int m = 0; m < M; ++m) {
+            float* w = ws + ((size_t)warp * M + m) * REC;
+#pragma unroll
+            for (int jj = 0; jj < DPL; ++jj) w[d0 + jj] = run_o[m][jj];
+            if (lane == 0) { w[HD] = run_mx[m]; w[HD + 1] = run_sum[m]; }
         }
         consumer_sync();
         for (int idx = tid; idx < M * HD; idx += kCW * 32) {
@@ -1008,16 +946,11 @@ __device__ void commit_copy(const FusedArgs& a, const Prog& P) {
     for (int l = blockIdx.x; l < P.b; l += gridDim.x) {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(a.slots + (size_t)istar * a.slot_stride + (size_t)l * a.slot_layer_stride);
         uint16_t* pg = a.kv + (size_t)l * a.kv_layer_elems + (size_t)page * page_elems;
-        // slot: [K | V][H][hd]; page: K [H][64][hd], then V transposed [H][hd][64]
-        const uint16_t* src16 = reinterpret_cast<const uint16_t*>(src);
-        for (int w = tid; w < a.H * hw; w += kCW * 32) {
-            const int h = w / hw, j = w % hw;
-            uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)h * kPageTokens + (np % kPageTokens)) * a.hd);
+        for (int w = tid; w < 2 * a.H * hw; w += kCW * 32) {
+            const int kv = w / (a.H * hw), rem = w % (a.H * hw), h = rem / hw, j = rem % hw;
+            uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)(kv * a.H + h) * kPageTokens + (np % kPageTokens)) * a.hd);
             dst[j] = __ldcg(src + w);
         }
-        uint16_t* vpg = pg + (size_t)a.H * kPageTokens * a.hd;
-        for (int e = tid; e < a.H * a.hd; e += kCW * 32)
-            vpg[(size_t)e * kPageTokens + (np % kPageTokens)] = __ldcg(src16 + (size_t)a.H * a.hd + e);
     }
     if (blockIdx.x == gridDim.x - 1)
         for (int i = tid; i < a.D; i += kCW * 32) a.main.h[i] = __ldcg(a.br.h + (size_t)istar * a.Dp + i);

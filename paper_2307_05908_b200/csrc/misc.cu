@@ -122,15 +122,12 @@ __global__ void commit_kernel(const CommitArgs a) {
         for (int l = blockIdx.x; l < a.b; l += gridDim.x) {
             const uint32_t* src = reinterpret_cast<const uint32_t*>(a.slots + (size_t)istar * a.slot_stride + (size_t)l * a.slot_layer_stride);
             uint16_t* pg = a.kv + (size_t)l * a.kv_layer_stride + (size_t)page * page_elems;
-            // slot: [K | V][H][hd]; page: K [H][64][hd], then V transposed [H][hd][64]
-            for (int w = threadIdx.x; w < a.H * hw; w += blockDim.x) {
-                const int h = w / hw, j = w % hw;
-                uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)h * kPageTokens + (np % kPageTokens)) * a.hd);
+            // words: [kv][h][hd/2]
+            for (int w = threadIdx.x; w < 2 * a.H * hw; w += blockDim.x) {
+                const int kv = w / (a.H * hw), rem = w % (a.H * hw), h = rem / hw, j = rem % hw;
+                uint32_t* dst = reinterpret_cast<uint32_t*>(pg + ((size_t)(kv * a.H + h) * kPageTokens + (np % kPageTokens)) * a.hd);
                 dst[j] = src[w];
             }
-            const uint16_t* src16 = reinterpret_cast<const uint16_t*>(src) + (size_t)a.H * a.hd;
-            uint16_t* vpg = pg + (size_t)a.H * kPageTokens * a.hd;
-            for (int e = threadIdx.x; e < a.H * a.hd; e += blockDim.x) vpg[(size_t)e * kPageTokens + (np % kPageTokens)] = src16[e];
         }
         if (blockIdx.x == 0)
             for (int i = threadIdx.x; i < a.D; i += blockDim.x) a.h_main[i] = a.h_branch[(size_t)istar * a.ldh + i];

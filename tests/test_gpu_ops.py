@@ -165,14 +165,11 @@ def _attention_case(H, hd, n_prefix, M, seed, use_slots, permute):
     kc = bf16_bits(rng, (n_prefix, D), 1.0)
     vc = bf16_bits(rng, (n_prefix, D), 1.0)
     table = rng.permutation(n_pages).astype(np.int32) if permute else np.arange(n_pages, dtype=np.int32)
-    # page = K [H][64][hd] followed by V transposed [H][hd][64]
-    pages = np.zeros((n_pages, 2, H, 64 * hd), dtype=np.uint16)
+    pages = np.zeros((n_pages, 2, H, 64, hd), dtype=np.uint16)
     pages[:] = 0x7FC0      # NaN bits: positions that must never be read
-    pk = pages[:, 0].reshape(n_pages, H, 64, hd)
-    pv = pages[:, 1].reshape(n_pages, H, hd, 64)
     for t in range(n_prefix):
-        pk[table[t // 64], :, t % 64, :] = kc[t].reshape(H, hd)
-        pv[table[t // 64], :, :, t % 64] = vc[t].reshape(H, hd)
+        pages[table[t // 64], 0, :, t % 64, :] = kc[t].reshape(H, hd)
+        pages[table[t // 64], 1, :, t % 64, :] = vc[t].reshape(H, hd)
     qkv = rng.standard_normal((M, 3 * D)).astype(np.float32)
     lib = ppd.load()
     rope = torch.zeros(n_prefix + 1, hd // 2, 2, dtype=torch.float32, device=DEV)
@@ -188,9 +185,7 @@ def _attention_case(H, hd, n_prefix, M, seed, use_slots, permute):
         tails = slots.cpu().numpy().view(np.uint16)
     else:
         pg = pages_d.cpu().numpy().view(np.uint16).reshape(pages.shape)[table[n_prefix // 64]]
-        k_row = pg[0].reshape(H, 64, hd)[:, n_prefix % 64, :].reshape(D)
-        v_row = pg[1].reshape(H, hd, 64)[:, :, n_prefix % 64].reshape(D)
-        tails = np.stack([np.stack([k_row, v_row])] * M)
+        tails = np.stack([np.stack([pg[0, :, n_prefix % 64, :].reshape(D), pg[1, :, n_prefix % 64, :].reshape(D)])] * M)
     kcf, vcf = ppd_inputs.bf16_to_f32(kc).astype(np.float64), ppd_inputs.bf16_to_f32(vc).astype(np.float64)
     for m in range(M):
         q = oracle.rope(qkv[m, :D], H, hd, n_prefix, theta)
