@@ -81,6 +81,16 @@ def greedy_step_flops(s, ctx_len):
     return s.n_layers * (layer_bytes(s) + 4 * s.d_model * ctx_len) + head_bytes(s)
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return list(values)
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 # ------------------------------------------------------------------ clocks
 
 class ClockSampler:
@@ -286,10 +296,7 @@ def run_gpu(args, wl):
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3
 
-    if dist is not None:
-        t = torch.tensor([ppd_ms, greedy_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ppd_ms, greedy_ms, e2e_ms = t.tolist()
+    ppd_ms, greedy_ms, e2e_ms = max_over_ranks([ppd_ms, greedy_ms, e2e_ms], dist, "cuda")
 
     peak, peak_kind = measured_peaks()
     ctx_mid = P + W + K // 2

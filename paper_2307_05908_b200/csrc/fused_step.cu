@@ -46,11 +46,8 @@ struct Cfg {
     static constexpr int kStageBytes = kGOff + kRowX;
     // after the ring: barriers | union {attention warp states + merge staging, head merge staging} | head lists | flags
     static constexpr int kBarBytes = 256;
-    static constexpr int kQs = 0;                                        // q [8][128] f32
-    static constexpr int kTail = kQs + kMaxRows * 128 * 4;               // ktail, vtail [8][128] bf16
-    static constexpr int kSc = kTail + 2 * kMaxRows * 128 * 2;           // sc [8][68] f32
-    static constexpr int kStat = kSc + kMaxRows * 68 * 4;                // (max, sum)[8]
-    static constexpr int kMerge = kStat + 64;                            // [kMergeChunk][130] f32
+    static constexpr int kWs = 0;                                        // per-warp attention states [8 warps][MR][130] f32
+    static constexpr int kMerge = kWs + kCW * MR * 130 * 4;              // [kMergeChunk][130] f32
     static constexpr int kUnionAttn = kMerge + kMergeChunk * 130 * 4;
     static constexpr int kUnionHead = kHeadMaxCtas * 8 * 8;              // staged candidate lists
     static constexpr int kUnion = ((kUnionAttn > kUnionHead ? kUnionAttn : kUnionHead) + 255) / 256 * 256;
@@ -76,7 +73,10 @@ struct OpDesc {            // one matrix product of a phase, as seen by this CTA
 };
 
 struct AttnDesc {          // the attention items (head, KV page) of one lane in a phase, as seen by this CTA
-    int M, p, n_splits, s_tail, total, first_item;
+    // Items are numbered j = head * n_splits + page; CTA index c (after the lane's offset) owns the
+    // contiguous range [c*q, (c+1)*q), so its items belong to one head or two and are pre-merged
+    // inside the CTA; a head is covered by n_segs(head) consecutive CTAs.
+    int M, p, n_splits, s_tail, total, q, j0, j1, c_idx;
     const float* qkv;
     uint16_t* kv_layer;
     uint16_t* slots;       // this layer's slots (row m at + m*slot_stride) or nullptr = cache
@@ -190,7 +190,10 @@ __device__ void fill_attn(const FusedArgs& a, int layer, const LaneBuf& ln, int 
     t.n_splits = p / kPageTokens + 1;
     t.s_tail = p / kPageTokens;
     t.total = a.H * t.n_splits;
-    t.first_item = ((int)blockIdx.x - cta_off + G) % G;
+    t.q = (t.total + G - 1) / G;
+    t.c_idx = ((int)blockIdx.x - cta_off + G) % G;
+    t.j0 = min(t.total, t.c_idx * t.q);
+    t.j1 = min(t.total, t.j0 + t.q);
     t.qkv = ln.qkv;
     t.kv_layer = a.kv + (size_t)layer * a.kv_layer_elems;
     t.slots = branch ? a.slots + (size_t)layer * a.slot_layer_stride : nullptr;
@@ -255,7 +258,7 @@ __device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P,
             for (int ln = 0; ln < pd.n_ops; ++ln) {
                 const AttnDesc& t = pd.at[ln];
                 it.lane = ln;
-                for (int j = t.first_item; j < t.total; j += G) {
+                for (int j = t.j0; j < t.j1; ++j) {
                     it.h = j / t.n_splits;
                     it.s = j - it.h * t.n_splits;
                     it.n_valid = min(kPageTokens, t.p - it.s * kPageTokens);
@@ -643,181 +646,278 @@ __device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh,
 __device__ __forceinline__ float rot_lo(float x0, float x1, float2 cs) { return __fmaf_rn(x0, cs.x, -__fmul_rn(x1, cs.y)); }
 __device__ __forceinline__ float rot_hi(float x0, float x1, float2 cs) { return __fmaf_rn(x1, cs.x, __fmul_rn(x0, cs.y)); }
 
-// Attention items of one lane: (head, KV page) pairs dealt round-robin to the CTAs.  The K/V tile
-// and the raw q (and, for the page that receives the new token, the raw k and v) rows arrive
-// through the ring.  The eight warps share an item: positions are spread over the warps for the
-// scores, rows over the warps for the softmax statistics, dims over the threads for P.V.
+// Sum over the 32 lanes of 32 per-lane values at once: after the call lane t holds the total of
+// v[t].  31 shuffles instead of 160; the order of additions is a fixed butterfly.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int half = 16; half >= 1; half >>= 1) {
+        const bool upper = (lane & half) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float keep = upper ? v[i + half] : v[i];
+            const float send = upper ? v[i] : v[i + half];
+            v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, half);
+        }
+    }
+    return v[0];
+}
+
+// Attention of one lane: this CTA's contiguous range of (head, KV page) items, cut into segments
+// of one head.  K/V tiles and the raw q (and, for the page that receives the new token, the raw k
+// and v) rows arrive through the ring.
+//  - Each page is processed by ONE warp, so up to eight pages run side by side: lane j owns dims
+//    [j*DPL, (j+1)*DPL) of the head; the scores of 32 positions are reduced across lanes together
+//    (lane t ends up owning positions t and t+32); softmax statistics by shuffles; P.V with the
+//    probabilities broadcast from their owner lanes.
+//  - A warp folds its pages (local index w, w+8, ...) into a running (max, sum, P.V) in registers;
+//    the 8 warp states of a segment are merged through shared memory in warp order.
+//  - A head covered by one CTA is finished there.  Otherwise every covering CTA writes one record
+//    and the last one to register (atomic ticket, nobody waits) merges the records in CTA order.
+// The structure depends on the position and the grid only, never on M or on which rows share
+// the launch.
 template <int M, int HD, int MB>
 __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared& sh, int& it) {
     using C = Cfg<MB>;
-    constexpr int DPL = HD / 32, HALF = HD / 2;
+    constexpr int DPL = HD / 32, HALF = HD / 2, REC = HD + 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, H = a.H;
     int* err = a.state + S_ERR;
-    float* qs = reinterpret_cast<float*>(sh.un + C::kQs);
-    uint16_t* ktail = reinterpret_cast<uint16_t*>(sh.un + C::kTail);
-    uint16_t* vtail = ktail + kMaxRows * 128;
-    float* sc = reinterpret_cast<float*>(sh.un + C::kSc);
-    float* stat = reinterpret_cast<float*>(sh.un + C::kStat);
     const float sscale = 1.4426950408889634f / sqrtf((float)HD);
     const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
-    for (int j = t.first_item; j < t.total; j += G, ++it) {
-        const int h = j / t.n_splits, s = j % t.n_splits;
-        const int n_valid = min(kPageTokens, t.p - s * kPageTokens);
-        const bool tail = s == t.s_tail;
-        const int slot = it % C::kStages;
-        mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
-        const uint8_t* st = sh.ring + slot * C::kStageBytes;
-        const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
-        const uint16_t* vs = ks + kPageTokens * HD;
-        const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
-        for (int idx = tid; idx < M * HALF; idx += kCW * 32) {
-            const int m = idx / HALF, i = idx % HALF;
-            const float2 cs = __ldg(a.rope + (size_t)t.p * HALF + i);
-            const float q0 = qraw[m * HD + i], q1 = qraw[m * HD + i + HALF];
-            qs[m * HD + i] = rot_lo(q0, q1, cs);
-            qs[m * HD + i + HALF] = rot_hi(q0, q1, cs);
-            if (tail) {
-                const float* kr = qraw + (M + m) * HD;
-                const float* vr = qraw + (2 * M + m) * HD;
-                const uint16_t k0 = f32_to_bf16_bits(rot_lo(kr[i], kr[i + HALF], cs));
-                const uint16_t k1 = f32_to_bf16_bits(rot_hi(kr[i], kr[i + HALF], cs));
-                const uint16_t v0 = f32_to_bf16_bits(vr[i]);
-                const uint16_t v1 = f32_to_bf16_bits(vr[i + HALF]);
-                ktail[m * HD + i] = k0; ktail[m * HD + i + HALF] = k1;
-                vtail[m * HD + i] = v0; vtail[m * HD + i + HALF] = v1;
-                uint16_t *kd, *vd;
-                if (t.slots) {
-                    kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
-                    vd = kd + (size_t)H * HD;
-                } else {
-                    uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
-                    kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
-                    vd = kd + (size_t)H * kPageTokens * HD;
+    const float NEG = __int_as_float(0xFF800000);
+    float* ws = reinterpret_cast<float*>(sh.un + C::kWs);          // [warp][m][REC]
+    const int d0 = lane * DPL;
+    const bool lo = d0 < HALF;
+    const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
+    float2 cs[DPL];
+#pragma unroll
+    for (int jj = 0; jj < DPL; ++jj) cs[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
+
+    for (int jseg = t.j0; jseg < t.j1;) {
+        // segment: this CTA's items of one head
+        const int h = jseg / t.n_splits;
+        const int s_lo = jseg - h * t.n_splits;
+        const int s_hi = min(t.n_splits, s_lo + (t.j1 - jseg));
+        jseg += s_hi - s_lo;
+        // CTAs covering this head, and this CTA's rank among them
+        const int c_first = (h * t.n_splits) / t.q;
+        const int n_segs = ((h + 1) * t.n_splits - 1) / t.q - c_first + 1;
+        const int r = t.c_idx - c_first;
+        float run_mx[M], run_sum[M], run_o[M][DPL];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            run_mx[m] = NEG; run_sum[m] = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = 0.f;
+        }
+        for (int s = s_lo; s < s_hi; ++s, ++it) {
+            const int slot = it % C::kStages;
+            // Every warp waits for every stage, also the ones it does not process: a warp that ran
+            // ahead would otherwise release a later use of the same ring slot too early.
+            mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
+            if ((s - s_lo) % kCW == warp) {
+                const int n_valid = min(kPageTokens, t.p - s * kPageTokens);
+                const bool tail = s == t.s_tail;
+                const uint8_t* st = sh.ring + slot * C::kStageBytes;
+                const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
+                const uint16_t* vs = ks + kPageTokens * HD;
+                const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
+                const int cnt = n_valid + (tail ? 1 : 0);      // <= 64
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    float qr[DPL], kt[DPL], vt[DPL];
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) {
+                        const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
+                        qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
+                        kt[jj] = 0.f; vt[jj] = 0.f;
+                    }
+                    if (tail) {
+                        // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
+                        const float* kr = qraw + (M + m) * HD;
+                        const float* vr = qraw + (2 * M + m) * HD;
+                        uint16_t kb[DPL], vb[DPL];
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) {
+                            const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
+                            kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
+                            vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
+                            kt[jj] = bf16_bits_to_f32(kb[jj]);
+                            vt[jj] = bf16_bits_to_f32(vb[jj]);
+                        }
+                        uint16_t *kd, *vd;
+                        if (t.slots) {
+                            kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                            vd = kd + (size_t)H * HD;
+                        } else {
+                            uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
+                            kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
+                            vd = kd + (size_t)H * kPageTokens * HD;
+                        }
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
+                    }
+                    // scores in log2 units: lane t gets positions t and t+32
+                    float sc0 = NEG, sc1 = NEG;
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {
+                        if (blk * 32 < n_valid) {
+                            float part[32];
+#pragma unroll
+                            for (int tt = 0; tt < 32; ++tt) {
+                                const int pos = blk * 32 + tt;
+                                float kf[DPL];
+                                if constexpr (DPL == 4) {
+                                    const uint2 kk = *reinterpret_cast<const uint2*>(ks + pos * HD + lane * 4);
+                                    kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
+                                } else {
+                                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + pos * HD + lane * 2);
+                                    kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
+                                }
+                                float dsum = 0.f;
+#pragma unroll
+                                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kf[jj], dsum);
+                                part[tt] = dsum;       // rows >= n_valid hold stale bytes: masked below
+                            }
+                            const float tot = transpose_reduce32(part, lane) * sscale;
+                            const bool ok = blk * 32 + lane < n_valid;
+                            if (blk == 0) sc0 = ok ? tot : NEG; else sc1 = ok ? tot : NEG;
+                        }
+                    }
+                    if (tail) {
+                        float dsum = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
+                        dsum = warp_sum(dsum) * sscale;
+                        if (n_valid < 32) { if (lane == n_valid) sc0 = dsum; }
+                        else if (lane == n_valid - 32) sc1 = dsum;
+                    }
+                    const float mx = warp_max(fmaxf(sc0, sc1));
+                    const float p0 = lane < cnt ? exp2f(sc0 - mx) : 0.f;
+                    const float p1 = lane + 32 < cnt ? exp2f(sc1 - mx) : 0.f;
+                    const float sum = warp_sum(p0 + p1);
+                    // P.V over the cached positions in ascending order, then the new token
+                    float o[DPL];
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
+                    for (int tt = 0; tt < n_valid; ++tt) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, tt < 32 ? p0 : p1, tt & 31);
+                        if constexpr (DPL == 4) {
+                            const uint2 vv = *reinterpret_cast<const uint2*>(vs + tt * HD + lane * 4);
+                            o[0] = fmaf(pw, bf16_lo(vv.x), o[0]); o[1] = fmaf(pw, bf16_hi(vv.x), o[1]);
+                            o[2] = fmaf(pw, bf16_lo(vv.y), o[2]); o[3] = fmaf(pw, bf16_hi(vv.y), o[3]);
+                        } else {
+                            const uint32_t vv = *reinterpret_cast<const uint32_t*>(vs + tt * HD + lane * 2);
+                            o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
+                        }
+                    }
+                    if (tail) {
+                        const float pw = __shfl_sync(0xFFFFFFFFu, n_valid < 32 ? p0 : p1, n_valid & 31);
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
+                    }
+                    // fold this page into the warp's running state
+                    const float nm = fmaxf(run_mx[m], mx);
+                    const float wa = exp2f(run_mx[m] - nm), wb = exp2f(mx - nm);
+#pragma unroll
+                    for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = fmaf(o[jj], wb, __fmul_rn(run_o[m][jj], wa));
+                    run_sum[m] = fmaf(sum, wb, __fmul_rn(run_sum[m], wa));
+                    run_mx[m] = nm;
                 }
-                kd[i] = k0; kd[i + HALF] = k1;
-                vd[i] = v0; vd[i + HALF] = v1;
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+        }
+        // merge the warp states (warp order) through shared memory
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float* w = ws + ((size_t)warp * M + m) * REC;
+#pragma unroll
+            for (int jj = 0; jj < DPL; ++jj) w[d0 + jj] = run_o[m][jj];
+            if (lane == 0) { w[HD] = run_mx[m]; w[HD + 1] = run_sum[m]; }
         }
         consumer_sync();
-        float qr[M][DPL];
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-#pragma unroll
-            for (int jj = 0; jj < DPL; ++jj) qr[m][jj] = qs[m * HD + lane * DPL + jj];
-        for (int tt = warp; tt < n_valid; tt += kCW) {
-            float kf[DPL];
-            if constexpr (DPL == 4) {
-                const uint2 kk = *reinterpret_cast<const uint2*>(ks + tt * HD + lane * 4);
-                kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
-            } else {
-                const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + tt * HD + lane * 2);
-                kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
-            }
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                float dsum = 0.f;
-#pragma unroll
-                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[m][jj], kf[jj], dsum);
-                dsum = warp_sum(dsum);
-                if (lane == 0) sc[m * 68 + tt] = dsum * sscale;
-            }
-        }
-        if (tail) {
-            for (int m = warp; m < M; m += kCW) {
-                float dsum = 0.f;
-#pragma unroll
-                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[m][jj], bf16_bits_to_f32(ktail[m * HD + lane * DPL + jj]), dsum);
-                dsum = warp_sum(dsum);
-                if (lane == 0) sc[m * 68 + n_valid] = dsum * sscale;
-            }
-        }
-        consumer_sync();
-        const int cnt = n_valid + (tail ? 1 : 0);
-        for (int m = warp; m < M; m += kCW) {
-            const float NEG = __int_as_float(0xFF800000);
-            const float v0 = lane < cnt ? sc[m * 68 + lane] : NEG;
-            const float v1 = lane + 32 < cnt ? sc[m * 68 + lane + 32] : NEG;
-            const float mx = warp_max(fmaxf(v0, v1));
-            const float p0 = lane < cnt ? exp2f(v0 - mx) : 0.f;
-            const float p1 = lane + 32 < cnt ? exp2f(v1 - mx) : 0.f;
-            if (lane < cnt) sc[m * 68 + lane] = p0;
-            if (lane + 32 < cnt) sc[m * 68 + lane + 32] = p1;
-            const float sum = warp_sum(p0 + p1);
-            if (lane == 0) { stat[2 * m] = mx; stat[2 * m + 1] = sum; }
-        }
-        consumer_sync();
-        // P.V: thread (m, dim) pairs spread over all 256 threads
         for (int idx = tid; idx < M * HD; idx += kCW * 32) {
-            const int m = idx / HD, dim = idx - m * HD;
-            float o = 0.f;
-            for (int tt = 0; tt < n_valid; ++tt) o = fmaf(sc[m * 68 + tt], bf16_bits_to_f32(vs[tt * HD + dim]), o);
-            if (tail) o = fmaf(sc[m * 68 + n_valid], bf16_bits_to_f32(vtail[m * HD + dim]), o);
-            float* part = t.partial + (((size_t)m * H + h) * a.max_splits + s) * (HD + 2);
-            part[dim] = o;
-            if (dim == 0) { part[HD] = stat[2 * m]; part[HD + 1] = stat[2 * m + 1]; }
+            const int m = idx / HD, jd = idx - m * HD;
+            float mx = ws[(size_t)m * REC + HD], num = ws[(size_t)m * REC + jd], den = ws[(size_t)m * REC + HD + 1];   // warp 0
+#pragma unroll
+            for (int w = 1; w < kCW; ++w) {
+                const float* rec = ws + ((size_t)w * M + m) * REC;
+                const float ms = rec[HD];
+                const float nm = fmaxf(mx, ms);
+                const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
+                num = fmaf(rec[jd], wb, __fmul_rn(num, wa));
+                den = fmaf(rec[HD + 1], wb, __fmul_rn(den, wa));
+                mx = nm;
+            }
+            if (n_segs == 1) {
+                t.out[(size_t)m * a.Dp + h * HD + jd] = num / den;
+            } else {
+                float* rec = t.partial + (((size_t)m * H + h) * a.max_splits + r) * REC;
+                rec[jd] = num;
+                if (jd == 0) { rec[HD] = mx; rec[HD + 1] = den; }
+            }
         }
         consumer_sync();
-        if (lane == 0) mbar_arrive(&sh.empty[slot]);
     }
 }
 
-// After all items of the phase: one fence, then every item registers with its head's ticket; the
-// CTA that registers a head's last page merges that head's pages in ascending order.
+// After all items of the phase: one fence, then this CTA registers once with the ticket of every
+// head it shares with other CTAs; the CTA that registers last merges the head's records (one per
+// covering CTA) in CTA order.
 template <int M, int HD, int MB>
 __device__ void attn_merge(const FusedArgs& a, const AttnDesc& t, const Shared& sh) {
     using C = Cfg<MB>;
     constexpr int REC = HD + 2;
     const int tid = threadIdx.x;
-    const int G = gridDim.x, H = a.H;
+    const int H = a.H;
     float* stage = reinterpret_cast<float*>(sh.un + C::kMerge);
-    const int my_items = t.first_item < t.total ? (t.total - 1 - t.first_item) / G + 1 : 0;
-    for (int i0 = 0; i0 < my_items; i0 += 64) {
-        const int nb = min(64, my_items - i0);
-        if (tid < nb) {
-            const int j = t.first_item + (i0 + tid) * G;
-            sh.flags[tid] = (atomicAdd(&t.tickets[j / t.n_splits], 1) == t.n_splits - 1) ? j / t.n_splits : -1;
-        }
+    for (int jseg = t.j0; jseg < t.j1;) {
+        const int h = jseg / t.n_splits;
+        jseg = min(t.j1, (h + 1) * t.n_splits);
+        const int c_first = (h * t.n_splits) / t.q;
+        const int n_segs = ((h + 1) * t.n_splits - 1) / t.q - c_first + 1;
+        if (n_segs == 1) continue;        // finished inside this CTA
+        if (tid == 0) sh.flags[0] = atomicAdd(&t.tickets[h], 1) == n_segs - 1;
         consumer_sync();
-        for (int q = 0; q < nb; ++q) {
-            const int h = sh.flags[q];
-            if (h < 0) continue;
-            __threadfence();
-            for (int m = 0; m < M; ++m) {
-                const float* part = t.partial + ((size_t)m * H + h) * a.max_splits * REC;
-                float mx = __int_as_float(0xFF800000), num = 0.f, den = 0.f;
-                for (int s0 = 0; s0 < t.n_splits; s0 += kMergeChunk) {
-                    const int ns = min(kMergeChunk, t.n_splits - s0);
-                    const int len = ns * REC;
-                    constexpr int LPT = (kMergeChunk * REC + 255) / 256;
-                    float tmp[LPT];
+        const bool last = sh.flags[0] != 0;
+        consumer_sync();
+        if (!last) continue;
+        __threadfence();
+        for (int m = 0; m < M; ++m) {
+            const float* part = t.partial + ((size_t)m * H + h) * a.max_splits * REC;
+            float mx = __int_as_float(0xFF800000), num = 0.f, den = 0.f;
+            for (int s0 = 0; s0 < n_segs; s0 += kMergeChunk) {
+                const int ns = min(kMergeChunk, n_segs - s0);
+                const int len = ns * REC;
+                constexpr int LPT = (kMergeChunk * REC + 255) / 256;
+                float tmp[LPT];
 #pragma unroll
-                    for (int u = 0; u < LPT; ++u) {
-                        const int c = tid + u * 256;
-                        tmp[u] = c < len ? __ldcg(part + (size_t)s0 * REC + c) : 0.f;
-                    }
-                    consumer_sync();
+                for (int u = 0; u < LPT; ++u) {
+                    const int c = tid + u * 256;
+                    tmp[u] = c < len ? __ldcg(part + (size_t)s0 * REC + c) : 0.f;
+                }
+                consumer_sync();
 #pragma unroll
-                    for (int u = 0; u < LPT; ++u) {
-                        const int c = tid + u * 256;
-                        if (c < len) stage[c] = tmp[u];
-                    }
-                    consumer_sync();
-                    if (tid < HD) {
-                        for (int s = 0; s < ns; ++s) {
-                            const float ms = stage[s * REC + HD];
-                            const float nm = fmaxf(mx, ms);
-                            const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
-                            num = fmaf(stage[s * REC + tid], wb, __fmul_rn(num, wa));
-                            den = fmaf(stage[s * REC + HD + 1], wb, __fmul_rn(den, wa));
-                            mx = nm;
-                        }
+                for (int u = 0; u < LPT; ++u) {
+                    const int c = tid + u * 256;
+                    if (c < len) stage[c] = tmp[u];
+                }
+                consumer_sync();
+                if (tid < HD) {
+                    for (int s = 0; s < ns; ++s) {
+                        const float ms = stage[s * REC + HD];
+                        const float nm = fmaxf(mx, ms);
+                        const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
+                        num = fmaf(stage[s * REC + tid], wb, __fmul_rn(num, wa));
+                        den = fmaf(stage[s * REC + HD + 1], wb, __fmul_rn(den, wa));
+                        mx = nm;
                     }
                 }
-                if (tid < HD) t.out[(size_t)m * a.Dp + h * HD + tid] = num / den;
             }
-            if (tid == 0) t.tickets[h] = 0;
+            if (tid < HD) t.out[(size_t)m * a.Dp + h * HD + tid] = num / den;
         }
+        if (tid == 0) t.tickets[h] = 0;
         consumer_sync();
     }
 }

@@ -207,6 +207,28 @@ def test_7b_shaped_two_layers_against_oracle(fused):
     check_against_oracle(shape, blob, prompt, 5, 3, 1, max_k=3, fused=fused)
 
 
+def test_13b_shaped_two_layers_against_oracle():
+    # shapes of the 13B workload (D 5120 = 20 column chunks, 40 heads, F 13824 = 54 chunks), 2 layers
+    shape = ppd_inputs.LLAMA_13B.with_layers(2)
+    blob = ppd_inputs.gen_weights(shape, seed=0)
+    prompt = ppd_inputs.gen_prompt(shape.vocab, 5, seed=1)
+    check_against_oracle(shape, blob, prompt, 4, 5, 1, max_k=5)
+
+
+def test_context_beyond_one_merge_round(tiny_shape, tiny_blob):
+    # 18 KV pages: more than one staging round of the page merge, ragged last page
+    prompt = ppd_inputs.gen_prompt(tiny_shape.vocab, 1100, seed=11)
+    ctx = ppd.Context(tiny_shape, max_seq=1160, max_k=3)
+    ctx.load_weights(tiny_blob)
+    check_against_oracle(tiny_shape, tiny_blob, prompt, 6, 3, 2, ctx=ctx, max_k=3)
+    ctx.prefill(prompt)
+    g, _ = ctx.decode(0, 0, 40)
+    ctx.prefill(prompt)
+    p, _ = ctx.decode(3, 3, 40)           # crosses the page boundary at 1152
+    assert (p == g).all()
+    ctx.close()
+
+
 def test_modes_agree_and_can_be_switched(tiny_shape, tiny_blob, tiny_prompt):
     ctx = ppd.Context(tiny_shape, max_seq=96, max_k=5)
     ctx.load_weights(tiny_blob)
