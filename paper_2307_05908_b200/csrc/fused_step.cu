@@ -99,6 +99,12 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
     return v;
 }
 
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 __device__ Prog build_prog(const FusedArgs& a) {
@@ -368,7 +374,8 @@ __device__ void producer_x(const FusedArgs& a, const Prog& P, uint8_t* smem, uin
     // wait in the CTA ends and the kernel terminates (outputs are then invalid).
     auto poll = [&]() {
         if (open >= P.n_phases - 1) return;
-        bool opened = ld_acquire_u64(cnt) >= base + (unsigned long long)(open + 1) * G;
+        bool opened = ld_relaxed_u64(cnt) >= base + (unsigned long long)(open + 1) * G;
+        if (opened) __threadfence();
         if (!opened) {
             const uint64_t now = global_timer_ns();
             if (t_idle == 0) t_idle = now;
@@ -1027,8 +1034,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
     int it = 0;
     PhaseDesc pd;
     for (int ph = 0; ph < P.n_phases; ++ph) {
+        make_phase(a, P, ph, MB, pd);        // overlaps the barrier latency
         mbar_wait(sh.phase_bar, ph & 1, err, kErrPhaseWait);
-        make_phase(a, P, ph, MB, pd);
         const bool trace = a.timeline && tid == 0 && ph < a.timeline_phases && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1);
         unsigned long long* tl = a.timeline + ((size_t)(blockIdx.x == 0 ? 0 : 1) * a.timeline_phases + ph) * 2;
         if (trace) tl[0] = global_timer_ns();
@@ -1073,10 +1080,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
         }
         // grid barrier arrival: everything this CTA wrote in the phase is visible before the count moves
         if (trace) tl[1] = global_timer_ns();
-        // the CTA barrier orders every consumer's writes before thread 0's fence (cumulativity)
+        // the CTA barrier orders every consumer's writes before thread 0's release (cumulativity)
         consumer_sync();
         if (tid == 0) {
-            __threadfence();
             asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(cnt) : "memory");
         }
     }
