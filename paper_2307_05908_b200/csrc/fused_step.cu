@@ -722,7 +722,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
             // Every warp waits for every stage, also the ones it does not process: a warp that ran
             // ahead would otherwise release a later use of the same ring slot too early.
             mbar_wait(&sh.full[slot], (it / C::kStages) & 1, err, kErrFullWait);
-            if ((s - s_lo) % kCW == warp) {
+            {
                 const int n_valid = min(kPageTokens, t.p - s * kPageTokens);
                 const bool tail = s == t.s_tail;
                 const uint8_t* st = sh.ring + slot * C::kStageBytes;
@@ -732,6 +732,10 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                 const int cnt = n_valid + (tail ? 1 : 0);      // <= 64
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
+                    // work unit = (page, row): page i of the segment, row m -> warp (i + m) % 8, so the
+                    // rows of one page spread over the warps.  For every row the pages a warp folds
+                    // together are those with the same i % 8, whatever M is.
+                    if (((s - s_lo) + m) % kCW != warp) continue;
                     float qr[DPL], kt[DPL], vt[DPL];
 #pragma unroll
                     for (int jj = 0; jj < DPL; ++jj) {
@@ -846,10 +850,12 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
         consumer_sync();
         for (int idx = tid; idx < M * HD; idx += kCW * 32) {
             const int m = idx / HD, jd = idx - m * HD;
-            float mx = ws[(size_t)m * REC + HD], num = ws[(size_t)m * REC + jd], den = ws[(size_t)m * REC + HD + 1];   // warp 0
+            // page groups c = 0..7 (pages i with i % 8 == c) in order; group c of row m sits in warp (c + m) % 8
+            const float* rec0 = ws + ((size_t)(m % kCW) * M + m) * REC;
+            float mx = rec0[HD], num = rec0[jd], den = rec0[HD + 1];
 #pragma unroll
-            for (int w = 1; w < kCW; ++w) {
-                const float* rec = ws + ((size_t)w * M + m) * REC;
+            for (int c = 1; c < kCW; ++c) {
+                const float* rec = ws + ((size_t)((c + m) % kCW) * M + m) * REC;
                 const float ms = rec[HD];
                 const float nm = fmaxf(mx, ms);
                 const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
