@@ -672,12 +672,12 @@ __device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane) {
 // Attention of one lane: this CTA's contiguous range of (head, KV page) items, cut into segments
 // of one head.  K/V tiles and the raw q (and, for the page that receives the new token, the raw k
 // and v) rows arrive through the ring.
-//  - Each page is processed by ONE warp, so up to eight pages run side by side: lane j owns dims
-//    [j*DPL, (j+1)*DPL) of the head; the scores of 32 positions are reduced across lanes together
-//    (lane t ends up owning positions t and t+32); softmax statistics by shuffles; P.V with the
-//    probabilities broadcast from their owner lanes.
-//  - A warp folds its pages (local index w, w+8, ...) into a running (max, sum, P.V) in registers;
-//    the 8 warp states of a segment are merged through shared memory in warp order.
+//  - Each (half page of 32 positions, row) is processed by ONE warp, so a few pages already keep
+//    all eight warps busy: lane j owns dims [j*DPL, (j+1)*DPL) of the head; the 32 scores are
+//    reduced across lanes together (lane t ends up owning position t); softmax statistics by
+//    shuffles; P.V with the probabilities broadcast from their owner lanes.
+//  - A warp folds its units into a running (max, sum, P.V) per row in registers; the 8 warp states
+//    of a segment are merged through shared memory in a fixed group order.
 //  - A head covered by one CTA is finished there.  Otherwise every covering CTA writes one record
 //    and the last one to register (atomic ticket, nobody waits) merges the records in CTA order.
 // The structure depends on the position and the grid only, never on M or on which rows share
@@ -729,54 +729,57 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                 const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
                 const uint16_t* vs = ks + kPageTokens * HD;
                 const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
-                const int cnt = n_valid + (tail ? 1 : 0);      // <= 64
 #pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    // work unit = (page, row): page i of the segment, row m -> warp (i + m) % 8, so the
-                    // rows of one page spread over the warps.  For every row the pages a warp folds
-                    // together are those with the same i % 8, whatever M is.
-                    if (((s - s_lo) + m) % kCW != warp) continue;
-                    float qr[DPL], kt[DPL], vt[DPL];
+                for (int hf = 0; hf < 2; ++hf) {
 #pragma unroll
-                    for (int jj = 0; jj < DPL; ++jj) {
-                        const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
-                        qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
-                        kt[jj] = 0.f; vt[jj] = 0.f;
-                    }
-                    if (tail) {
-                        // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
-                        const float* kr = qraw + (M + m) * HD;
-                        const float* vr = qraw + (2 * M + m) * HD;
-                        uint16_t kb[DPL], vb[DPL];
+                    for (int m = 0; m < M; ++m) {
+                        // Work unit = (half page, row): unit u = 2 * page + half of the segment, row m ->
+                        // warp (u + m) % 8, so the halves and rows of one page spread over the warps.  For
+                        // every row the units a warp folds together are those with the same u % 8,
+                        // whatever M is.
+                        if ((2 * (s - s_lo) + hf + m) % kCW != warp) continue;
+                        const int nv = min(32, n_valid - 32 * hf);              // cached positions in this half
+                        const bool has_new = tail && (n_valid >> 5) == hf;     // the new token falls into this half
+                        if (nv <= 0 && !has_new) continue;
+                        float qr[DPL], kt[DPL], vt[DPL];
 #pragma unroll
                         for (int jj = 0; jj < DPL; ++jj) {
-                            const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
-                            kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
-                            vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
-                            kt[jj] = bf16_bits_to_f32(kb[jj]);
-                            vt[jj] = bf16_bits_to_f32(vb[jj]);
+                            const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
+                            qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
+                            kt[jj] = 0.f; vt[jj] = 0.f;
                         }
-                        uint16_t *kd, *vd;
-                        if (t.slots) {
-                            kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
-                            vd = kd + (size_t)H * HD;
-                        } else {
-                            uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
-                            kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
-                            vd = kd + (size_t)H * kPageTokens * HD;
+                        if (has_new) {
+                            // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
+                            const float* kr = qraw + (M + m) * HD;
+                            const float* vr = qraw + (2 * M + m) * HD;
+                            uint16_t kb[DPL], vb[DPL];
+#pragma unroll
+                            for (int jj = 0; jj < DPL; ++jj) {
+                                const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
+                                kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
+                                vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
+                                kt[jj] = bf16_bits_to_f32(kb[jj]);
+                                vt[jj] = bf16_bits_to_f32(vb[jj]);
+                            }
+                            uint16_t *kd, *vd;
+                            if (t.slots) {
+                                kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                                vd = kd + (size_t)H * HD;
+                            } else {
+                                uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
+                                kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
+                                vd = kd + (size_t)H * kPageTokens * HD;
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
                         }
-#pragma unroll
-                        for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
-                    }
-                    // scores in log2 units: lane t gets positions t and t+32
-                    float sc0 = NEG, sc1 = NEG;
-#pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-                        if (blk * 32 < n_valid) {
+                        // scores in log2 units: lane t gets position 32*hf + t; the new token takes lane nv
+                        float sc = NEG;
+                        if (nv > 0) {
                             float part[32];
 #pragma unroll
                             for (int tt = 0; tt < 32; ++tt) {
-                                const int pos = blk * 32 + tt;
+                                const int pos = hf * 32 + tt;
                                 float kf[DPL];
                                 if constexpr (DPL == 4) {
                                     const uint2 kk = *reinterpret_cast<const uint2*>(ks + pos * HD + lane * 4);
@@ -788,52 +791,52 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                                 float dsum = 0.f;
 #pragma unroll
                                 for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kf[jj], dsum);
-                                part[tt] = dsum;       // rows >= n_valid hold stale bytes: masked below
+                                part[tt] = dsum;       // rows >= nv hold stale bytes: masked below
                             }
                             const float tot = transpose_reduce32(part, lane) * sscale;
-                            const bool ok = blk * 32 + lane < n_valid;
-                            if (blk == 0) sc0 = ok ? tot : NEG; else sc1 = ok ? tot : NEG;
+                            sc = lane < nv ? tot : NEG;
                         }
-                    }
-                    if (tail) {
-                        float dsum = 0.f;
+                        const int nvp = nv > 0 ? nv : 0;
+                        if (has_new) {
+                            float dsum = 0.f;
 #pragma unroll
-                        for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
-                        dsum = warp_sum(dsum) * sscale;
-                        if (n_valid < 32) { if (lane == n_valid) sc0 = dsum; }
-                        else if (lane == n_valid - 32) sc1 = dsum;
-                    }
-                    const float mx = warp_max(fmaxf(sc0, sc1));
-                    const float p0 = lane < cnt ? exp2f(sc0 - mx) : 0.f;
-                    const float p1 = lane + 32 < cnt ? exp2f(sc1 - mx) : 0.f;
-                    const float sum = warp_sum(p0 + p1);
-                    // P.V over the cached positions in ascending order, then the new token
-                    float o[DPL];
-#pragma unroll
-                    for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
-                    for (int tt = 0; tt < n_valid; ++tt) {
-                        const float pw = __shfl_sync(0xFFFFFFFFu, tt < 32 ? p0 : p1, tt & 31);
-                        if constexpr (DPL == 4) {
-                            const uint2 vv = *reinterpret_cast<const uint2*>(vs + tt * HD + lane * 4);
-                            o[0] = fmaf(pw, bf16_lo(vv.x), o[0]); o[1] = fmaf(pw, bf16_hi(vv.x), o[1]);
-                            o[2] = fmaf(pw, bf16_lo(vv.y), o[2]); o[3] = fmaf(pw, bf16_hi(vv.y), o[3]);
-                        } else {
-                            const uint32_t vv = *reinterpret_cast<const uint32_t*>(vs + tt * HD + lane * 2);
-                            o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
+                            for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
+                            dsum = warp_sum(dsum) * sscale;
+                            if (lane == nvp) sc = dsum;        // nvp <= 31: the tail page caches at most 63 positions
                         }
-                    }
-                    if (tail) {
-                        const float pw = __shfl_sync(0xFFFFFFFFu, n_valid < 32 ? p0 : p1, n_valid & 31);
+                        const int cnt = nvp + (has_new ? 1 : 0);
+                        const float mx = warp_max(sc);
+                        const float pr = lane < cnt ? exp2f(sc - mx) : 0.f;
+                        const float sum = warp_sum(pr);
+                        // P.V over the cached positions in ascending order, then the new token
+                        float o[DPL];
 #pragma unroll
-                        for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
-                    }
-                    // fold this page into the warp's running state
-                    const float nm = fmaxf(run_mx[m], mx);
-                    const float wa = exp2f(run_mx[m] - nm), wb = exp2f(mx - nm);
+                        for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
+                        for (int tt = 0; tt < nvp; ++tt) {
+                            const float pw = __shfl_sync(0xFFFFFFFFu, pr, tt);
+                            const int pos = hf * 32 + tt;
+                            if constexpr (DPL == 4) {
+                                const uint2 vv = *reinterpret_cast<const uint2*>(vs + pos * HD + lane * 4);
+                                o[0] = fmaf(pw, bf16_lo(vv.x), o[0]); o[1] = fmaf(pw, bf16_hi(vv.x), o[1]);
+                                o[2] = fmaf(pw, bf16_lo(vv.y), o[2]); o[3] = fmaf(pw, bf16_hi(vv.y), o[3]);
+                            } else {
+                                const uint32_t vv = *reinterpret_cast<const uint32_t*>(vs + pos * HD + lane * 2);
+                                o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
+                            }
+                        }
+                        if (has_new) {
+                            const float pw = __shfl_sync(0xFFFFFFFFu, pr, nvp);
 #pragma unroll
-                    for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = fmaf(o[jj], wb, __fmul_rn(run_o[m][jj], wa));
-                    run_sum[m] = fmaf(sum, wb, __fmul_rn(run_sum[m], wa));
-                    run_mx[m] = nm;
+                            for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
+                        }
+                        // fold this unit into the warp's running state
+                        const float nm = fmaxf(run_mx[m], mx);
+                        const float wa = exp2f(run_mx[m] - nm), wb = exp2f(mx - nm);
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) run_o[m][jj] = fmaf(o[jj], wb, __fmul_rn(run_o[m][jj], wa));
+                        run_sum[m] = fmaf(sum, wb, __fmul_rn(run_sum[m], wa));
+                        run_mx[m] = nm;
+                    }
                 }
             }
             __syncwarp();
@@ -850,7 +853,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
         consumer_sync();
         for (int idx = tid; idx < M * HD; idx += kCW * 32) {
             const int m = idx / HD, jd = idx - m * HD;
-            // page groups c = 0..7 (pages i with i % 8 == c) in order; group c of row m sits in warp (c + m) % 8
+            // unit groups c = 0..7 (units u with u % 8 == c) in order; group c of row m sits in warp (c + m) % 8
             const float* rec0 = ws + ((size_t)(m % kCW) * M + m) * REC;
             float mx = rec0[HD], num = rec0[jd], den = rec0[HD + 1];
 #pragma unroll
