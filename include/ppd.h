@@ -83,6 +83,15 @@ void ppd_destroy(ppd_ctx* ctx);
  * nearest-even).  bytes must equal the blob size for cfg. */
 int ppd_load_weights(ppd_ctx* ctx, const void* host_blob, size_t bytes, int dtype);
 
+/* Gives the early head a classifier of its own (Table 2, column "Y": a language-modelling
+ * classifier trained for the intermediate layer with the rest of the model frozen; Section 4.3).
+ * The early logits become W_E . RMSNorm_final(h_l); the final head keeps W_H, so the token stream
+ * is unchanged and only the match rate moves.  host_w: host, [vocab][d_model] row-major, dtype as
+ * in ppd_load_weights, may be freed on return.  dev_mem: device, caller-owned, 256-byte aligned,
+ * >= ppd_packed_bytes(vocab, d_model) bytes, kept alive while the classifier is in use.
+ * host_w = NULL returns to the shared classifier (column "N").  Needs loaded weights. */
+int ppd_load_early_head(ppd_ctx* ctx, const void* host_w, size_t bytes, int dtype, void* dev_mem, size_t dev_bytes);
+
 /* ---------------------------------------------------------------- decoding */
 
 /* Fills the KV cache from a prompt (host, n_prompt >= 1 ids in [0, vocab)).  The last prompt

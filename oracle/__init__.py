@@ -55,6 +55,8 @@ def _load():
         "orc_embed": (None, [_P, _I, _P]),
         "orc_layer": (None, [_P, _I, _P, _I, _I]),
         "orc_head": (None, [_P, _P, _P]),
+        "orc_early_head": (None, [_P, _P, _P]),
+        "orc_set_early_head": (None, [_P, _P]),
         "orc_rmsnorm": (None, [_P, _P, _I, _D, _P]),
         "orc_matvec": (None, [_P, _I, _I, _P, _P]),
         "orc_rope": (None, [_P, _I, _I, _I, _D]),
@@ -225,6 +227,19 @@ class Oracle:
         h = _f64(h).copy()
         self._lib.orc_layer(self._m, layer, _ptr(h), pos, slot)
         return h
+
+    def set_early_head(self, w_bf16):
+        """Classifier of the early head: uint16 (bf16) [vocab][d_model], or None for the shared one."""
+        self._early = None if w_bf16 is None else np.ascontiguousarray(w_bf16, dtype=np.uint16)   # kept alive
+        if self._early is not None:
+            assert self._early.shape == (self.shape.vocab, self.shape.d_model)
+        self._lib.orc_set_early_head(self._m, _ptr(self._early))
+
+    def early_head(self, h):
+        h = _f64(h)
+        out = np.empty(self.shape.vocab, dtype=np.float64)
+        self._lib.orc_early_head(self._m, _ptr(h), _ptr(out))
+        return out
 
     def head(self, h):
         h = _f64(h)

@@ -47,6 +47,7 @@ typedef struct orc_model {
     const uint16_t* emb;
     const uint16_t* g_final;
     const uint16_t* w_head;
+    const uint16_t* w_early;  /* classifier of the early head; the final one unless replaced */
     orc_layer_w* lw;
     double *kc, *vc;  /* canonical cache  [layer][max_seq][D] */
     double *kb, *vb;  /* branch slots     [max_k][layer][D]   */
@@ -201,6 +202,7 @@ orc_model* orc_create(const orc_config* c, const uint16_t* blob) {
     }
     m->g_final = p; p += D;
     m->w_head = p;
+    m->w_early = p;
     size_t cache = (size_t)c->n_layers * (size_t)c->max_seq * D;
     size_t slots = (size_t)(c->max_k > 0 ? c->max_k : 1) * (size_t)c->n_layers * D;
     m->kc = (double*)calloc(cache, sizeof(double));
@@ -287,17 +289,24 @@ void orc_layer(orc_model* m, int layer, double* h, int pos, int slot) {
     m->t_layers += now_s() - t0;
 }
 
-/* logits = W_H . RMSNorm_final(h).  Used for the final head and, unchanged, for the early
- * head (the untrained-classifier variant of the paper's Table 2, column "N"). */
-void orc_head(orc_model* m, const double* h, double* logits) {
+/* logits = W . RMSNorm_final(h).  The final head uses the model's unembedding W_H.  The early
+ * head uses the same W_H by default (the paper's Table 2, column "N": the classifier trained
+ * for the final layer applied at an intermediate one) or a classifier of its own (column "Y":
+ * trained for that layer with everything else frozen), see orc_set_early_head. */
+static void head_with(orc_model* m, const uint16_t* w, const double* h, double* logits) {
     double t0 = now_s();
     int D = m->c.d_model;
     double* n = (double*)malloc(sizeof(double) * D);
     orc_rmsnorm(h, m->g_final, D, m->c.rms_eps, n);
-    orc_matvec(m->w_head, m->c.vocab, D, n, logits);
+    orc_matvec(w, m->c.vocab, D, n, logits);
     free(n);
     m->t_heads += now_s() - t0;
 }
+void orc_head(orc_model* m, const double* h, double* logits) { head_with(m, m->w_head, h, logits); }
+void orc_early_head(orc_model* m, const double* h, double* logits) { head_with(m, m->w_early, h, logits); }
+
+/* w: bf16 [vocab][d_model], borrowed; NULL restores the shared classifier. */
+void orc_set_early_head(orc_model* m, const uint16_t* w) { m->w_early = w ? w : m->w_head; }
 
 /* gap between the r-th and (r+1)-th largest logits (r counted from 1) */
 static double margin_at(const double* logits, int V, int r) {
@@ -354,7 +363,7 @@ int orc_greedy_probe(orc_model* m, int32_t n, int32_t k, int32_t l, const int32_
         orc_embed(m, m->pending, h);
         for (int j = 0; j < d; ++j) {
             orc_layer(m, j, h, m->pos, -1);
-            if (j + 1 == l && k > 0) orc_head(m, h, le);
+            if (j + 1 == l && k > 0) orc_early_head(m, h, le);
         }
         orc_head(m, h, lf);
         int32_t next;
@@ -419,7 +428,7 @@ int orc_ppd(orc_model* m, int32_t n, int32_t k, int32_t l, int32_t eos, int32_t*
             for (int j = b; j < l; ++j) orc_layer(m, j, h, pos, -1);
             u += l - b;
         }
-        orc_head(m, h, lg);
+        orc_early_head(m, h, lg);
         orc_topk(lg, V, k, cand);
         for (int i = 0; i < k; ++i) {
             double* hi = hb + (size_t)i * D;

@@ -47,6 +47,7 @@ SIGNATURES = {
     "ppd_create": (ctypes.c_int, [_CFG, _P, _SZ, _P, _P, ctypes.POINTER(_P)]),
     "ppd_destroy": (None, [_P]),
     "ppd_load_weights": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int]),
+    "ppd_load_early_head": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int, _P, _SZ]),
     "ppd_prefill": (ctypes.c_int, [_P, _P, _I]),
     "ppd_greedy_step": (ctypes.c_int, [_P, _P]),
     "ppd_decode": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P]),
@@ -157,6 +158,23 @@ class Context:
         dtype = {np.dtype(np.uint16): 1, np.dtype(np.float32): 0}[blob.dtype]
         with self._dev():
             _check(self.lib.ppd_load_weights(self._h, blob.ctypes.data, blob.nbytes, dtype), self._h)
+
+    def load_early_head(self, w):
+        """w: uint16 (bf16) or float32 [vocab][d_model] classifier for the early head, or None to share
+        the final head's.  The packed copy lives in a torch buffer owned by this context."""
+        if w is None:
+            with self._dev():
+                _check(self.lib.ppd_load_early_head(self._h, None, 0, 1, None, 0), self._h)
+            self._early_buf = None
+            return
+        w = np.ascontiguousarray(w)
+        dtype = {np.dtype(np.uint16): 1, np.dtype(np.float32): 0}[w.dtype]
+        nbytes = self.lib.ppd_packed_bytes(self.shape.vocab, self.shape.d_model)
+        with self._dev():
+            buf = self._torch.empty(nbytes + 256, dtype=self._torch.uint8, device=self.device)
+            base = (buf.data_ptr() + 255) // 256 * 256
+            _check(self.lib.ppd_load_early_head(self._h, w.ctypes.data, w.nbytes, dtype, base, nbytes), self._h)
+        self._early_buf = buf
 
     def prefill(self, prompt):
         p = np.ascontiguousarray(prompt, dtype=np.int32)

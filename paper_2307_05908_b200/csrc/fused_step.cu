@@ -221,7 +221,7 @@ __device__ void make_phase(const FusedArgs& a, const Prog& P, int ph, int MB, Ph
         if (lb >= 0) { fill_attn(a, lb, a.br, MB, P.pos + 1, true, G / 2, pd.at[1]); pd.n_ops = 2; }
     } else if (pd.kind == PH_HEAD_EARLY || pd.kind == PH_HEAD_FINAL) {
         OpDesc& o = pd.op[0];
-        o.w = a.w_head; o.N = a.V; o.K = a.D; o.x = a.main.h; o.ldx = a.Dp; o.gain = a.g_final; o.resid = nullptr;
+        o.w = pd.kind == PH_HEAD_EARLY ? a.w_head_early : a.w_head; o.N = a.V; o.K = a.D; o.x = a.main.h; o.ldx = a.Dp; o.gain = a.g_final; o.resid = nullptr;
         o.mode = kHead; o.out = pd.kind == PH_HEAD_EARLY ? a.logits_early : a.logits_final; o.ldo = a.V; o.M = 1;
         o.n_rg = (o.N + kTileRows - 1) / kTileRows;
         o.n_kc = (o.K + kTileCols - 1) / kTileCols;

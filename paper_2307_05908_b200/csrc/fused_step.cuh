@@ -30,6 +30,7 @@ struct FusedArgs {
     const uint16_t* emb;
     const float* g_final;
     const uint16_t* w_head;
+    const uint16_t* w_head_early;   // classifier of the early head (== w_head unless one was loaded)
     // KV cache
     uint16_t* kv;
     long long kv_layer_elems;

@@ -138,6 +138,7 @@ struct ppd_ctx {
     Lane lane[2];
     int* state;
     bool trace;                       // record per-phase timestamps of the fused kernel
+    const uint16_t* w_early;          // packed classifier of the early head in caller memory, or nullptr = W_H
     bool fused;                       // true: one persistent kernel per step; false: per-op kernels on two streams
     std::vector<cudaEvent_t> step_ev; // per-step timing events of the fused path (grown on demand)
     std::vector<int32_t> h_tokens;    // staging for the bulk read-back
@@ -209,13 +210,13 @@ int run_layers(ppd_ctx* x, int lane_id, int M, int l0, int l1, const int* d_pos,
 }
 
 // logits = W_H . RMSNorm_final(h of the main lane); top-8 into `top` (ids at +0, values at +32 ints)
-int run_head(ppd_ctx* x, size_t logits_off, size_t top_off, cudaStream_t st) {
+int run_head(ppd_ctx* x, size_t logits_off, size_t top_off, cudaStream_t st, bool early = false) {
     const ppd_config& c = x->c;
     const Layout& L = x->L;
     GemvArgs g{};
     g.err = x->state + S_ERR;
     g.eps = c.rms_eps;
-    g.w = at<uint16_t>(x, L.w_head); g.N = c.vocab; g.K = c.d_model;
+    g.w = (early && x->w_early) ? x->w_early : at<uint16_t>(x, L.w_head); g.N = c.vocab; g.K = c.d_model;
     g.x = x->lane[0].h; g.ldx = L.Dp; g.gain = at<float>(x, L.g_final);
     g.out = at<float>(x, logits_off); g.ldo = c.vocab;
     g.head_scratch = at<void>(x, L.head_scratch);
@@ -302,7 +303,7 @@ int decode_step(ppd_ctx* x, int k, int l, int32_t* token, uint8_t* hit) {
     } else {
         b = l < d - l ? l : d - l;
         if ((rc = run_layers(x, 0, 1, start, l, d_pos, 0, false, x->sm))) return rc;
-        if ((rc = run_head(x, L.logits_early, L.top_early, x->sm))) return rc;
+        if ((rc = run_head(x, L.logits_early, L.top_early, x->sm, true))) return rc;
         CK(cudaEventRecord(x->ev_early, x->sm));
         // candidate branches: k rows through layers 1..b at position pos+1
         CK(cudaStreamWaitEvent(x->sb, x->ev_early, 0));
@@ -348,6 +349,7 @@ void fill_fused(ppd_ctx* x, FusedArgs& f) {
     f.off_wqkv = (long long)L.off_wqkv; f.off_wo = (long long)L.off_wo; f.off_wgu = (long long)L.off_wgu;
     f.off_wd = (long long)L.off_wd; f.off_g1 = (long long)L.off_g1; f.off_g2 = (long long)L.off_g2;
     f.emb = at<uint16_t>(x, L.emb); f.g_final = at<float>(x, L.g_final); f.w_head = at<uint16_t>(x, L.w_head);
+    f.w_head_early = x->w_early ? x->w_early : f.w_head;
     f.kv = at<uint16_t>(x, L.kv); f.kv_layer_elems = L.kv_layer_elems; f.page_table = at<int>(x, L.page_table);
     f.slots = at<uint16_t>(x, L.slots); f.slot_stride = L.slot_elems; f.slot_layer_stride = L.slot_layer_elems;
     f.rope = at<float2>(x, L.rope); f.max_splits = L.max_splits;
@@ -495,6 +497,7 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     x->loaded = x->prefilled = false;
     x->pdl = true;
     x->fused = true;
+    x->w_early = nullptr;
     x->trace = false;
     x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
     x->cuda_err = cudaSuccess;
@@ -604,6 +607,33 @@ int ppd_load_weights(ppd_ctx* x, const void* host_blob, size_t bytes, int dtype)
     CK(cudaStreamSynchronize(x->sm));
     x->loaded = true;
     x->prefilled = false;
+    return PPD_OK;
+}
+
+int ppd_load_early_head(ppd_ctx* x, const void* host_w, size_t bytes, int dtype, void* dev_mem, size_t dev_bytes) {
+    if (!x) return PPD_EINVAL;
+    if (!host_w) {                     // back to the shared classifier
+        CK(cudaStreamSynchronize(x->sm));
+        x->w_early = nullptr;
+        return PPD_OK;
+    }
+    if (dtype != 0 && dtype != 1) return PPD_EINVAL;
+    if (!x->loaded) return PPD_ESTATE;
+    const size_t V = x->c.vocab, D = x->c.d_model, es = dtype == 0 ? 4 : 2;
+    if (bytes != V * D * es || !dev_mem || ((uintptr_t)dev_mem % kAlign) != 0) return PPD_EINVAL;
+    if (dev_bytes < ppd_packed_bytes((int)V, (int)D)) return PPD_ENOSPC;
+    uint16_t* dst = reinterpret_cast<uint16_t*>(dev_mem);
+    uint8_t* staging = x->base + x->L.staging;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(host_w);
+    CK(cudaMemsetAsync(dst, 0, ppd_packed_bytes((int)V, (int)D), x->sm));
+    const size_t max_rows = kStagingBytes / (D * es);
+    for (size_t r0 = 0; r0 < V; r0 += max_rows) {
+        const size_t nr = V - r0 < max_rows ? V - r0 : max_rows;
+        CK(cudaMemcpyAsync(staging, src + r0 * D * es, nr * D * es, cudaMemcpyHostToDevice, x->sm));
+        CK(launch_pack(staging, dtype == 0, (int)nr, (int)D, dst, 1, (int)r0, x->sm));
+    }
+    CK(cudaStreamSynchronize(x->sm));
+    x->w_early = dst;
     return PPD_OK;
 }
 

@@ -229,6 +229,43 @@ def test_context_beyond_one_merge_round(tiny_shape, tiny_blob):
     ctx.close()
 
 
+@pytest.mark.parametrize("fused", [True, False], ids=["fused", "per-op"])
+def test_separate_early_classifier(tiny_shape, tiny_blob, tiny_prompt, fused):
+    """A classifier of its own for the early head (Table 2 column "Y"): tokens unchanged, early logits
+    and hit flags follow the replaced classifier, parity with the oracle given the same classifier."""
+    rng = np.random.default_rng(3)
+    w_h = ppd_inputs.blob_views(tiny_shape, tiny_blob)["W_H"]
+    w_e = w_h.copy()
+    rows = rng.choice(tiny_shape.vocab, tiny_shape.vocab * 3 // 10, replace=False)
+    w_e[rows] = ppd_inputs.gen_weights(tiny_shape, seed=77)[: w_h.size].reshape(w_h.shape)[rows]
+    n, k, l = 16, 3, 2
+    ctx = ppd.Context(tiny_shape, max_seq=64, max_k=k)
+    ctx.set_mode(fused)
+    ctx.load_weights(tiny_blob)
+    ctx.prefill(tiny_prompt)
+    base_t, base_h = ctx.decode(k, l, n)
+    ctx.load_early_head(w_e)
+    o = Oracle(tiny_shape, tiny_blob, max_seq=64, max_k=k)
+    o.set_early_head(w_e)
+    o.prefill(tiny_prompt)
+    ref = o.greedy_probe(n, k=k, l=l, dump_logits=True)
+    ctx.prefill(tiny_prompt)
+    toks, hits, fl, el, cands = gpu_stream(ctx, k, l, n, forced=ref["tokens"])
+    assert np.abs(el - ref["early_logits"]).max() < LOGIT_TOL and np.abs(fl - ref["final_logits"]).max() < LOGIT_TOL
+    for s_ in range(n):
+        assert (cands[s_] == oracle_topk(el[s_], k)).all() and hits[s_] == int(toks[s_] in cands[s_])
+    safe = (ref["margin_final"] > MARGIN) & (ref["margin_early"] > MARGIN)
+    assert (hits[safe] == ref["hit"][safe]).all()
+    ctx.prefill(tiny_prompt)
+    t2, h2 = ctx.decode(k, l, n)
+    assert (t2 == base_t).all()                      # exactness does not depend on the classifier
+    ctx.load_early_head(None)
+    ctx.prefill(tiny_prompt)
+    t3, h3 = ctx.decode(k, l, n)
+    assert (t3 == base_t).all() and (h3 == base_h).all()
+    ctx.close()
+
+
 def test_modes_agree_and_can_be_switched(tiny_shape, tiny_blob, tiny_prompt):
     ctx = ppd.Context(tiny_shape, max_seq=96, max_k=5)
     ctx.load_weights(tiny_blob)

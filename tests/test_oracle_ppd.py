@@ -124,3 +124,36 @@ def test_argument_checks(tiny_shape, tiny_blob, tiny_prompt):
         o.ppd(4, 3, 0)                       # early layer out of range
     with pytest.raises(ValueError):
         o.ppd(20, 3, 2)                      # cache would overflow
+
+
+def test_separate_early_classifier(tiny_shape, tiny_blob, tiny_prompt):
+    """Table 2 column "Y": the early head may use a classifier of its own.  Exactness does not
+    depend on it; the match flags follow the replaced classifier."""
+    rng = np.random.default_rng(3)
+    w_h = ppd_inputs.blob_views(tiny_shape, tiny_blob)["W_H"]
+    # a classifier correlated with the final one (stand-in for a trained head): W_H with 30% of its rows redrawn
+    w_e = w_h.copy()
+    rows = rng.choice(tiny_shape.vocab, tiny_shape.vocab * 3 // 10, replace=False)
+    w_e[rows] = ppd_inputs.gen_weights(tiny_shape, seed=77)[: tiny_shape.vocab * tiny_shape.d_model].reshape(w_h.shape)[rows]
+    o = Oracle(tiny_shape, tiny_blob, max_seq=64)
+    o.prefill(tiny_prompt)
+    base = o.greedy_probe(16, k=3, l=2, dump_logits=True)
+    o.set_early_head(w_e)
+    o.prefill(tiny_prompt)
+    g = o.greedy_probe(16, k=3, l=2, dump_logits=True)
+    o.prefill(tiny_prompt)
+    p = o.ppd(16, 3, 2)
+    assert (g["tokens"] == base["tokens"]).all() and (p["tokens"] == base["tokens"]).all()     # exact whatever the head
+    assert (p["hit"] == g["hit"]).all()
+    assert np.allclose(g["final_logits"], base["final_logits"])
+    assert not np.allclose(g["early_logits"], base["early_logits"])
+    # untouched vocabulary rows give the same early logits, redrawn rows differ
+    keep = np.setdiff1d(np.arange(tiny_shape.vocab), rows)
+    assert np.allclose(g["early_logits"][:, keep], base["early_logits"][:, keep])
+    # hits are defined by the replaced classifier's top-k
+    for s_ in range(16):
+        top = np.lexsort((np.arange(tiny_shape.vocab), -g["early_logits"][s_]))[:3]
+        assert g["hit"][s_] == int(g["tokens"][s_] in top)
+    o.set_early_head(None)
+    o.prefill(tiny_prompt)
+    assert (o.greedy_probe(16, k=3, l=2)["hit"] == base["hit"]).all()
