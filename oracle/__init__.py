@@ -57,6 +57,8 @@ def _load():
         "orc_head": (None, [_P, _P, _P]),
         "orc_early_head": (None, [_P, _P, _P]),
         "orc_set_early_head": (None, [_P, _P]),
+        "orc_set_sampling": (ctypes.c_int, [_P, _I, _D, _P, _I]),
+        "orc_sample_topk": (_I, [_P, _I, _I, _D, _D]),
         "orc_rmsnorm": (None, [_P, _P, _I, _D, _P]),
         "orc_matvec": (None, [_P, _I, _I, _P, _P]),
         "orc_rope": (None, [_P, _I, _I, _I, _D]),
@@ -136,6 +138,12 @@ def topk(logits, k):
     ids = np.empty(k, dtype=np.int32)
     lib.orc_topk(_ptr(lg), lg.size, k, _ptr(ids))
     return ids
+
+
+def sample_topk(logits, ks, temperature, u):
+    """Top-k sampling of one token: softmax(logits / T) over the ks largest, inverse CDF at u."""
+    lg = _f64(logits)
+    return _load().orc_sample_topk(_ptr(lg), lg.size, ks, float(temperature), float(u))
 
 
 def round_bf16(x):
@@ -227,6 +235,15 @@ class Oracle:
         h = _f64(h).copy()
         self._lib.orc_layer(self._m, layer, _ptr(h), pos, slot)
         return h
+
+    def set_sampling(self, ks, temperature=1.0, u=None):
+        """Final prediction by top-k sampling over ks tokens (0 = greedy); u[pos] in [0,1) is used for the
+        token fed at position pos."""
+        self._u = None if u is None else _f64(u)      # kept alive: the C side borrows it
+        rc = self._lib.orc_set_sampling(self._m, ks, float(temperature), _ptr(self._u),
+                                        0 if self._u is None else self._u.size)
+        if rc != 0:
+            raise ValueError("bad sampling parameters")
 
     def set_early_head(self, w_bf16):
         """Classifier of the early head: uint16 (bf16) [vocab][d_model], or None for the shared one."""

@@ -48,6 +48,10 @@ typedef struct orc_model {
     const uint16_t* g_final;
     const uint16_t* w_head;
     const uint16_t* w_early;  /* classifier of the early head; the final one unless replaced */
+    int32_t sample_k;         /* 0: greedy final prediction; >= 1: top-k sampling over this many tokens */
+    double temperature;
+    const double* sample_u;   /* uniform numbers in [0,1), one per position (index = position of the fed token) */
+    int32_t n_sample_u;
     orc_layer_w* lw;
     double *kc, *vc;  /* canonical cache  [layer][max_seq][D] */
     double *kb, *vb;  /* branch slots     [max_k][layer][D]   */
@@ -170,6 +174,29 @@ void orc_topk(const double* logits, int V, int k, int32_t* ids) {
     }
 }
 
+/*
+ * Top-k sampling of the final prediction (Appendix B: PPD with a sampled instead of a greedy
+ * final prediction; Fan et al.'s top-k sampling): keep the ks largest logits in the order
+ * (value descending, id ascending), p_i = softmax(logit_i / T) over them, and return the first
+ * token whose cumulative probability exceeds u (the last one if rounding leaves none).
+ * ks = 1 is the argmax.
+ */
+int32_t orc_sample_topk(const double* logits, int V, int ks, double T, double u) {
+    int32_t ids[64];
+    double w[64];
+    if (ks > 64) ks = 64;
+    if (ks > V) ks = V;
+    orc_topk(logits, V, ks, ids);
+    double tot = 0.0;
+    for (int i = 0; i < ks; ++i) { w[i] = exp((logits[ids[i]] - logits[ids[0]]) / T); tot += w[i]; }
+    double acc = 0.0;
+    for (int i = 0; i < ks; ++i) {
+        acc += w[i] / tot;
+        if (u < acc) return ids[i];
+    }
+    return ids[ks - 1];
+}
+
 /* ------------------------------------------------------------------ model */
 
 size_t orc_blob_elems(const orc_config* c) {
@@ -218,6 +245,23 @@ orc_model* orc_create(const orc_config* c, const uint16_t* blob) {
 void orc_destroy(orc_model* m) {
     if (!m) return;
     free(m->kc); free(m->vc); free(m->kb); free(m->vb); free(m->lw); free(m);
+}
+
+/* Final prediction by top-k sampling (ks >= 1, temperature T > 0) with the given uniform numbers,
+ * u[pos] being used for the token fed at position pos; ks = 0 returns to greedy.  u is borrowed. */
+int orc_set_sampling(orc_model* m, int32_t ks, double T, const double* u, int32_t n_u) {
+    if (ks < 0 || ks > 64 || (ks > 0 && (!(T > 0.0) || !u || n_u < 1))) return -1;
+    m->sample_k = ks; m->temperature = T; m->sample_u = u; m->n_sample_u = n_u;
+    return 0;
+}
+
+/* the final prediction for the token fed at position pos */
+static int32_t final_prediction(const orc_model* m, const double* logits, int pos) {
+    if (m->sample_k > 0 && pos < m->n_sample_u)
+        return orc_sample_topk(logits, m->c.vocab, m->sample_k, m->temperature, m->sample_u[pos]);
+    int32_t next;
+    orc_topk(logits, m->c.vocab, 1, &next);
+    return next;
 }
 
 void orc_reset(orc_model* m) { m->pos = 0; m->pending = -1; m->t_layers = m->t_heads = 0.0; }
@@ -366,8 +410,7 @@ int orc_greedy_probe(orc_model* m, int32_t n, int32_t k, int32_t l, const int32_
             if (j + 1 == l && k > 0) orc_early_head(m, h, le);
         }
         orc_head(m, h, lf);
-        int32_t next;
-        orc_topk(lf, V, 1, &next);
+        const int32_t next = final_prediction(m, lf, m->pos);
         tokens[s] = next;
         if (k > 0) {
             orc_topk(le, V, k, ids);
@@ -439,8 +482,7 @@ int orc_ppd(orc_model* m, int32_t n, int32_t k, int32_t l, int32_t eos, int32_t*
         for (int j = l; j < d; ++j) orc_layer(m, j, h, pos, -1);
         u += d - l;
         orc_head(m, h, lg);
-        int32_t next;
-        orc_topk(lg, V, 1, &next);
+        const int32_t next = final_prediction(m, lg, pos);
         int istar = -1;
         for (int i = 0; i < k; ++i) if (cand[i] == next) istar = i;
         if (istar >= 0) {

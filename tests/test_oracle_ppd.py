@@ -157,3 +157,64 @@ def test_separate_early_classifier(tiny_shape, tiny_blob, tiny_prompt):
     o.set_early_head(None)
     o.prefill(tiny_prompt)
     assert (o.greedy_probe(16, k=3, l=2)["hit"] == base["hit"]).all()
+
+
+def test_topk_sampling_rule():
+    """Appendix B: the final prediction may be sampled.  Pins of the sampling rule itself."""
+    import math
+    import oracle
+    lg = np.array([0.3, 2.0, -1.0, 1.5, 2.0, 0.0])
+    # ks = 1 is the argmax (lowest id on ties), whatever u
+    assert all(oracle.sample_topk(lg, 1, 0.7, u) == 1 for u in (0.0, 0.5, 0.999999))
+    # two candidates: closed form p(first) = 1 / (1 + exp(-(l0 - l1)/T))
+    two = np.array([1.0, 0.25, -5.0])
+    for T in (0.5, 1.0, 2.0):
+        p0 = 1.0 / (1.0 + math.exp(-(1.0 - 0.25) / T))
+        assert oracle.sample_topk(two, 2, T, p0 - 1e-9) == 0 and oracle.sample_topk(two, 2, T, p0 + 1e-9) == 1
+    # inverse CDF over the candidate order (value descending, id ascending): ids 1, 4, 3 for ks = 3
+    w = np.exp(np.array([2.0, 2.0, 1.5]) - 2.0)
+    cdf = np.cumsum(w / w.sum())
+    for u, want in ((0.0, 1), (cdf[0] - 1e-9, 1), (cdf[0] + 1e-9, 4), (cdf[1] + 1e-9, 3), (0.999999999, 3)):
+        assert oracle.sample_topk(lg, 3, 1.0, u) == want
+    # frequencies over a fine grid of u follow the softmax of the kept logits; nothing else is drawn
+    us = (np.arange(20000) + 0.5) / 20000
+    draws = np.array([oracle.sample_topk(lg, 3, 1.0, u) for u in us])
+    assert set(draws) == {1, 3, 4}
+    for i, tok in enumerate((1, 4, 3)):
+        assert abs((draws == tok).mean() - w[i] / w.sum()) < 1e-4
+    # low temperature concentrates on the best token
+    assert (np.array([oracle.sample_topk(lg, 3, 0.01, u) for u in us[::100]]) != 3).all()
+
+
+def test_ppd_with_sampled_final_prediction_is_exact(tiny_shape, tiny_blob, tiny_prompt):
+    """PPD with a sampled final prediction gives the same stream as plain sampling with the same
+    random numbers (Appendix B), and differs from the greedy stream."""
+    n = 24
+    rng = np.random.default_rng(5)
+    u = rng.random(128)
+    o = Oracle(tiny_shape, tiny_blob, max_seq=64)
+    o.prefill(tiny_prompt)
+    greedy = o.greedy_probe(n, k=3, l=2)
+    o.set_sampling(3, 1.0, u)
+    o.prefill(tiny_prompt)
+    plain = o.greedy_probe(n, k=3, l=2, dump_logits=True)
+    for k, l in ((1, 1), (3, 2), (5, 3)):
+        o.prefill(tiny_prompt)
+        g = o.greedy_probe(n, k=k, l=l)
+        o.prefill(tiny_prompt)
+        p = o.ppd(n, k, l)
+        assert (p["tokens"] == plain["tokens"]).all() and (g["tokens"] == plain["tokens"]).all()
+        assert (p["hit"] == g["hit"]).all()
+    assert (plain["tokens"] != greedy["tokens"]).any()
+    # every drawn token is one of the three best of that step's final logits, chosen by u[position]
+    pos0 = len(tiny_prompt) - 1
+    for s_ in range(n):
+        import oracle as orc
+        assert plain["tokens"][s_] == orc.sample_topk(plain["final_logits"][s_], 3, 1.0, u[pos0 + s_])
+    # sampling over one token is greedy decoding
+    o.set_sampling(1, 1.0, u)
+    o.prefill(tiny_prompt)
+    assert (o.greedy_probe(n)["tokens"] == greedy["tokens"]).all()
+    o.set_sampling(0)
+    o.prefill(tiny_prompt)
+    assert (o.ppd(n, 3, 2)["tokens"] == greedy["tokens"]).all()
