@@ -92,6 +92,15 @@ int ppd_load_weights(ppd_ctx* ctx, const void* host_blob, size_t bytes, int dtyp
  * host_w = NULL returns to the shared classifier (column "N").  Needs loaded weights. */
 int ppd_load_early_head(ppd_ctx* ctx, const void* host_w, size_t bytes, int dtype, void* dev_mem, size_t dev_bytes);
 
+/* Sampled final prediction (Appendix B: PPD applies unchanged when the final prediction is drawn by
+ * top-k sampling instead of taken as the argmax; the early candidates stay the early head's top-k).
+ * top_k in 1..8: the token fed at position pos is followed by the first of the top_k best final
+ * logits (order: value descending, id ascending) whose cumulative softmax(logit / temperature)
+ * exceeds u[pos]; positions >= n_u fall back to the argmax.  top_k = 0 restores greedy decoding.
+ * u: host, n_u <= max_seq values in [0, 1), copied.  Applies to ppd_greedy_step, ppd_decode and
+ * ppd_step alike, so PPD and plain decoding draw the same stream from the same numbers. */
+int ppd_set_sampling(ppd_ctx* ctx, int32_t top_k, float temperature, const float* u, int32_t n_u);
+
 /* ---------------------------------------------------------------- decoding */
 
 /* Fills the KV cache from a prompt (host, n_prompt >= 1 ids in [0, vocab)).  The last prompt

@@ -48,6 +48,7 @@ SIGNATURES = {
     "ppd_destroy": (None, [_P]),
     "ppd_load_weights": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int]),
     "ppd_load_early_head": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int, _P, _SZ]),
+    "ppd_set_sampling": (ctypes.c_int, [_P, _I, _F, _P, _I]),
     "ppd_prefill": (ctypes.c_int, [_P, _P, _I]),
     "ppd_greedy_step": (ctypes.c_int, [_P, _P]),
     "ppd_decode": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P]),
@@ -175,6 +176,12 @@ class Context:
             base = (buf.data_ptr() + 255) // 256 * 256
             _check(self.lib.ppd_load_early_head(self._h, w.ctypes.data, w.nbytes, dtype, base, nbytes), self._h)
         self._early_buf = buf
+
+    def set_sampling(self, top_k, temperature=1.0, u=None):
+        """Top-k sampling of the final prediction (0 = greedy); u[pos] in [0,1) per position, float32."""
+        uu = None if u is None else np.ascontiguousarray(u, dtype=np.float32)
+        with self._dev():
+            _check(self.lib.ppd_set_sampling(self._h, top_k, temperature, _np_ptr(uu), 0 if uu is None else uu.size), self._h)
 
     def prefill(self, prompt):
         p = np.ascontiguousarray(prompt, dtype=np.int32)

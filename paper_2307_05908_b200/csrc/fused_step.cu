@@ -954,7 +954,7 @@ __device__ void run_attn_merge(const FusedArgs& a, const AttnDesc& t, const Shar
 // pos+1 and its hidden state becomes the main one.  CTA c copies layers c, c+G, ...
 __device__ void commit_copy(const FusedArgs& a, const Prog& P) {
     if (P.mode != kPpdStep) return;
-    const int token = __ldcg(a.top_final);
+    const int token = pick_token(a.top_final, a.sample_k, a.temperature, a.sample_u, a.n_sample_u, P.pos);
     int istar = -1;
     for (int i = 0; i < P.k; ++i)
         if (__ldcg(a.top_early + i) == token) istar = i;
@@ -982,7 +982,7 @@ __device__ void state_update(const FusedArgs& a, const Prog& P) {
     unsigned long long* base = reinterpret_cast<unsigned long long*>(a.state + S_BAR_BASE);
     *base = *base + (unsigned long long)P.n_phases * gridDim.x;
     if (P.mode == kPrefillToken) return;
-    const int token = __ldcg(a.top_final);
+    const int token = pick_token(a.top_final, a.sample_k, a.temperature, a.sample_u, a.n_sample_u, P.pos);
     int istar = -1;
     if (P.mode == kPpdStep)
         for (int i = 0; i < P.k; ++i)

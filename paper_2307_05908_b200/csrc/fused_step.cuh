@@ -49,6 +49,11 @@ struct FusedArgs {
     float *logits_early, *logits_final;
     int *top_early, *top_final;   // ids[8]; values (float) at +32 words
     void* head_scratch;
+    // sampled final prediction (top-k sampling over the best sample_k <= 8 tokens; 0 = argmax)
+    int sample_k;
+    float temperature;
+    const float* sample_u;   // uniform numbers, index = position of the fed token
+    int n_sample_u;
     // state and outputs
     int* state;
     int* out_tokens;
@@ -57,6 +62,24 @@ struct FusedArgs {
     unsigned long long* timeline;   // optional: [cta in {0, last}][phase][start, end] in ns; nullptr = off
     int timeline_phases;            // capacity in phases
 };
+
+// The final prediction from the head's ordered top-8 list: the argmax, or, with top-k sampling
+// (Appendix B of the paper), the first of the best `ks` tokens whose cumulative softmax(logit / T)
+// exceeds u.  Plain float arithmetic in a fixed order: every caller gets the same token.
+__device__ __forceinline__ int pick_token(const int* top, int ks, float T, const float* u_arr, int n_u, int pos) {
+    const float* vals = reinterpret_cast<const float*>(top) + 32;
+    if (ks <= 0 || pos >= n_u) return __ldcg(top);
+    const float u = __ldg(u_arr + pos);
+    const float v0 = __ldcg(vals);
+    float w[8], tot = 0.f;
+    for (int i = 0; i < ks; ++i) { w[i] = expf((__ldcg(vals + i) - v0) / T); tot += w[i]; }
+    float acc = 0.f;
+    for (int i = 0; i < ks; ++i) {
+        acc += w[i] / tot;
+        if (u < acc) return __ldcg(top + i);
+    }
+    return __ldcg(top + ks - 1);
+}
 
 // Launches the step kernel for `mb` branch rows (0 = no branches: prefill token or greedy step).
 cudaError_t launch_fused_step(const FusedArgs& a, int mb, cudaStream_t st, bool pdl, int n_sms);

@@ -2,6 +2,7 @@
 // and PPD's verify/commit step.
 #include "common.cuh"
 #include "misc.cuh"
+#include "fused_step.cuh"
 
 namespace ppd {
 
@@ -109,11 +110,11 @@ __global__ void commit_kernel(const CommitArgs a) {
     pdl_launch_dependents();
     pdl_wait();
     __shared__ int s_last;
-    const int token = a.final_ids[0];
+    const int pos = *a.d_pos;
+    const int token = pick_token(a.final_ids, a.sample_k, a.temperature, a.sample_u, a.n_sample_u, pos);
     int istar = -1;
     for (int i = 0; i < a.k; ++i)
         if (a.cand[i] == token) istar = i;
-    const int pos = *a.d_pos;
     if (istar >= 0) {
         const int np = pos + 1;
         const int page = a.page_table[np / kPageTokens];

@@ -29,6 +29,10 @@ struct CommitArgs {
     uint8_t* out_hit;         // [max_steps]
     float* out_margin;        // [max_steps] top-1 minus top-2 final logit
     int* last;                // [2] (token, hit) of this step
+    int sample_k;             // top-k sampling of the final prediction (0 = argmax)
+    float temperature;
+    const float* sample_u;
+    int n_sample_u;
 };
 
 cudaError_t launch_embed(const uint16_t* E, const int* tokens, int M, int D, float* h, int ldh, cudaStream_t st, bool pdl);

@@ -35,7 +35,7 @@ struct Layout {
     size_t ws[2];            // main / branch workspaces
     size_t ws_h, ws_qkv, ws_attn, ws_z, ws_part, ws_tick, ws_bytes[2];   // offsets inside a workspace
     size_t logits_final, logits_early, top_final, top_early, head_scratch;
-    size_t state, prompt, out_tokens, out_hit, out_margin, timeline, staging, total;
+    size_t state, sample_u, prompt, out_tokens, out_hit, out_margin, timeline, staging, total;
 };
 
 bool valid_config(const ppd_config* c) {
@@ -104,6 +104,7 @@ Layout plan(const ppd_config& c) {
     L.top_early = take(64 * 4);
     L.head_scratch = take(kHeadScratchBytes);
     L.state = take(256);
+    L.sample_u = take((size_t)c.max_seq * 4);
     L.prompt = take((size_t)c.max_seq * 4);
     L.out_tokens = take((size_t)c.max_seq * 4);
     L.out_hit = take((size_t)c.max_seq);
@@ -138,6 +139,8 @@ struct ppd_ctx {
     Lane lane[2];
     int* state;
     bool trace;                       // record per-phase timestamps of the fused kernel
+    int sample_k, n_sample_u;         // top-k sampling of the final prediction (0 = greedy)
+    float temperature;
     const uint16_t* w_early;          // packed classifier of the early head in caller memory, or nullptr = W_H
     bool fused;                       // true: one persistent kernel per step; false: per-op kernels on two streams
     std::vector<cudaEvent_t> step_ev; // per-step timing events of the fused path (grown on demand)
@@ -243,6 +246,7 @@ int run_commit(ppd_ctx* x, int k, int b, cudaStream_t st) {
     a.ticket = x->state + S_TICKET;
     a.out_tokens = at<int>(x, L.out_tokens); a.out_hit = at<uint8_t>(x, L.out_hit); a.out_margin = at<float>(x, L.out_margin);
     a.last = x->state + S_LAST_TOKEN;
+    a.sample_k = x->sample_k; a.temperature = x->temperature; a.sample_u = at<float>(x, L.sample_u); a.n_sample_u = x->n_sample_u;
     CK(launch_commit(a, st, x->pdl));
     x->stats.kernel_launches += 1;
     return PPD_OK;
@@ -361,6 +365,7 @@ void fill_fused(ppd_ctx* x, FusedArgs& f) {
     f.logits_early = at<float>(x, L.logits_early); f.logits_final = at<float>(x, L.logits_final);
     f.top_early = at<int>(x, L.top_early); f.top_final = at<int>(x, L.top_final);
     f.head_scratch = at<void>(x, L.head_scratch);
+    f.sample_k = x->sample_k; f.temperature = x->temperature; f.sample_u = at<float>(x, L.sample_u); f.n_sample_u = x->n_sample_u;
     f.state = x->state;
     f.out_tokens = at<int>(x, L.out_tokens); f.out_hit = at<uint8_t>(x, L.out_hit); f.out_margin = at<float>(x, L.out_margin);
     f.timeline = x->trace ? at<unsigned long long>(x, L.timeline) : nullptr;
@@ -498,6 +503,7 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     x->pdl = true;
     x->fused = true;
     x->w_early = nullptr;
+    x->sample_k = 0; x->n_sample_u = 0; x->temperature = 1.f;
     x->trace = false;
     x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
     x->cuda_err = cudaSuccess;
@@ -634,6 +640,23 @@ int ppd_load_early_head(ppd_ctx* x, const void* host_w, size_t bytes, int dtype,
     }
     CK(cudaStreamSynchronize(x->sm));
     x->w_early = dst;
+    return PPD_OK;
+}
+
+int ppd_set_sampling(ppd_ctx* x, int32_t top_k, float temperature, const float* u, int32_t n_u) {
+    if (!x || top_k < 0 || top_k > PPD_MAX_K) return PPD_EINVAL;
+    if (top_k > 0 && (!(temperature > 0.f) || !u || n_u < 1)) return PPD_EINVAL;
+    if (top_k > 0 && n_u > x->c.max_seq) return PPD_ENOSPC;
+    CK(cudaStreamSynchronize(x->sm));
+    if (top_k > 0) {
+        for (int i = 0; i < n_u; ++i)
+            if (!(u[i] >= 0.f && u[i] < 1.f)) return PPD_EINVAL;
+        CK(cudaMemcpyAsync(x->base + x->L.sample_u, u, (size_t)n_u * 4, cudaMemcpyHostToDevice, x->sm));
+        CK(cudaStreamSynchronize(x->sm));
+    }
+    x->sample_k = top_k;
+    x->temperature = top_k > 0 ? temperature : 1.f;
+    x->n_sample_u = top_k > 0 ? n_u : 0;
     return PPD_OK;
 }
 

@@ -266,6 +266,52 @@ def test_separate_early_classifier(tiny_shape, tiny_blob, tiny_prompt, fused):
     ctx.close()
 
 
+def test_sampled_final_prediction(tiny_ctx, tiny_shape, tiny_blob, tiny_prompt):
+    """Appendix B: with a top-k sampled final prediction PPD still reproduces plain decoding with the
+    same random numbers; every draw follows the rule on the library's own logits; parity with the
+    oracle where the draw is not within rounding of a boundary."""
+    import oracle as orc
+    n, ks, T = 24, 3, 1.0
+    u = np.random.default_rng(5).random(400).astype(np.float32)
+    try:
+        tiny_ctx.set_sampling(ks, T, u)
+        tiny_ctx.prefill(tiny_prompt)
+        plain, _, pfl, _, _ = gpu_stream(tiny_ctx, 0, 0, n)
+        for k, l in ((1, 1), (3, 2), (5, 3)):
+            tiny_ctx.prefill(tiny_prompt)
+            toks, hits, fl, el, cands = gpu_stream(tiny_ctx, k, l, n)
+            assert (toks == plain).all() and np.array_equal(fl, pfl)
+            for s_ in range(n):
+                assert hits[s_] == int(toks[s_] in cands[s_])
+        pos0 = len(tiny_prompt) - 1
+        o = Oracle(tiny_shape, tiny_blob, max_seq=64)
+        o.set_sampling(ks, T, u.astype(np.float64))
+        o.prefill(tiny_prompt)
+        ref = o.greedy_probe(n, k=3, l=2, forced=plain, dump_logits=True)
+        checked = 0
+        for s_ in range(n):
+            lg = pfl[s_].astype(np.float64)
+            top = orc.topk(lg, ks + 1)
+            w = np.exp((lg[top[:ks]] - lg[top[0]]) / T)
+            cdf = np.cumsum(w / w.sum())
+            if np.abs(cdf[:-1] - u[pos0 + s_]).min() < 1e-5:
+                continue                      # the draw sits on a boundary: float vs double may differ
+            assert plain[s_] == orc.sample_topk(lg, ks, T, float(u[pos0 + s_]))      # rule on own logits
+            checked += 1
+            if lg[top[ks - 1]] - lg[top[ks]] > MARGIN and np.abs(cdf[:-1] - u[pos0 + s_]).min() > 1e-2:
+                assert plain[s_] == ref["tokens"][s_]                                 # and the oracle's draw
+        assert checked >= n - 2
+        tiny_ctx.set_sampling(1, 1.0, u)          # one candidate: greedy
+        tiny_ctx.prefill(tiny_prompt)
+        g1, _ = tiny_ctx.decode(3, 2, n)
+        tiny_ctx.set_sampling(0)
+        tiny_ctx.prefill(tiny_prompt)
+        g0, _ = tiny_ctx.decode(3, 2, n)
+        assert (g1 == g0).all() and (g0 != plain).any()
+    finally:
+        tiny_ctx.set_sampling(0)
+
+
 def test_modes_agree_and_can_be_switched(tiny_shape, tiny_blob, tiny_prompt):
     ctx = ppd.Context(tiny_shape, max_seq=96, max_k=5)
     ctx.load_weights(tiny_blob)
