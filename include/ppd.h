@@ -105,8 +105,14 @@ int ppd_set_sampling(ppd_ctx* ctx, int32_t top_k, float temperature, const float
 
 /* Fills the KV cache from a prompt (host, n_prompt >= 1 ids in [0, vocab)).  The last prompt
  * token is the start token x_0 of Algorithm 1: positions 0..n_prompt-2 are cached and
- * prompt[n_prompt-1] stays pending for the first decode step.  Resets the position. */
+ * prompt[n_prompt-1] stays pending for the first decode step.  Resets the position.  In the default
+ * mode the prompt runs through the step kernel in chunks of 4 tokens per launch. */
 int ppd_prefill(ppd_ctx* ctx, const int32_t* prompt, int32_t n_prompt);
+
+/* Prompt tokens processed per prefill launch in the default mode: 4 (default), 8, 2 or 1.  The
+ * tokens of a chunk share one pass over the weights and attend causally to each other; chunk
+ * sizes differ in rounding only. */
+int ppd_set_prefill_chunk(ppd_ctx* ctx, int32_t n_tokens);
 
 /* One conventional greedy step: all d layers, argmax of the final logits (Section 1).
  * out_token: host, one id. */

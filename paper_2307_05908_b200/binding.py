@@ -49,6 +49,7 @@ SIGNATURES = {
     "ppd_load_weights": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int]),
     "ppd_load_early_head": (ctypes.c_int, [_P, _P, _SZ, ctypes.c_int, _P, _SZ]),
     "ppd_set_sampling": (ctypes.c_int, [_P, _I, _F, _P, _I]),
+    "ppd_set_prefill_chunk": (ctypes.c_int, [_P, _I]),
     "ppd_prefill": (ctypes.c_int, [_P, _P, _I]),
     "ppd_greedy_step": (ctypes.c_int, [_P, _P]),
     "ppd_decode": (ctypes.c_int, [_P, _I, _I, _I, _I, _P, _P, _P]),
@@ -176,6 +177,9 @@ class Context:
             base = (buf.data_ptr() + 255) // 256 * 256
             _check(self.lib.ppd_load_early_head(self._h, w.ctypes.data, w.nbytes, dtype, base, nbytes), self._h)
         self._early_buf = buf
+
+    def set_prefill_chunk(self, n_tokens):
+        _check(self.lib.ppd_set_prefill_chunk(self._h, n_tokens), self._h)
 
     def set_sampling(self, top_k, temperature=1.0, u=None):
         """Top-k sampling of the final prediction (0 = greedy); u[pos] in [0,1) per position, float32."""

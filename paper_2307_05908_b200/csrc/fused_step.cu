@@ -77,6 +77,7 @@ struct AttnDesc {          // the attention items (head, KV page) of one lane in
     // contiguous range [c*q, (c+1)*q), so its items belong to one head or two and are pre-merged
     // inside the CTA; a head is covered by n_segs(head) consecutive CTAs.
     int M, p, n_splits, s_tail, total, q, j0, j1, c_idx;
+    bool chunk;            // prefill chunk: row m sits at position p + m and also sees the new tokens of rows < m
     const float* qkv;
     uint16_t* kv_layer;
     uint16_t* slots;       // this layer's slots (row m at + m*slot_stride) or nullptr = cache
@@ -111,6 +112,14 @@ __device__ Prog build_prog(const FusedArgs& a) {
     Prog P;
     P.mode = a.mode; P.k = a.k; P.l = a.l; P.d = a.d;
     P.b = 0; P.start = 0;
+    if (a.mode == kPrefillChunk) {
+        // k consecutive prompt tokens as the k rows of the "branch" lane through all d layers; the main
+        // lane is idle.  Rows sit at positions pos .. pos+k-1 and attend causally inside the chunk.
+        P.pos = a.pos_val;
+        P.b = a.d; P.la = 0; P.n_seg_a = 0; P.n_fused = a.d; P.embed_main = 0;
+        P.n_phases = 1 + 5 * a.d + 1;
+        return P;
+    }
     if (a.mode == kPrefillToken) {
         P.pos = a.pos_val;
     } else {
@@ -132,6 +141,13 @@ __device__ Prog build_prog(const FusedArgs& a) {
 __device__ void phase_info(const Prog& P, int ph, int& kind, int& lm, int& lb) {
     lm = lb = -1;
     int q = ph;
+    if (P.mode == kPrefillChunk) {
+        if (q == 0) { kind = PH_EMBED_BR; return; }
+        --q;
+        if (q < 5 * P.d) { kind = PH_QKV + q % 5; lb = q / 5; return; }
+        kind = PH_STATE;
+        return;
+    }
     if (P.embed_main) {
         if (q == 0) { kind = PH_EMBED_MAIN; return; }
         --q;
@@ -200,9 +216,10 @@ __device__ void fill_attn(const FusedArgs& a, int layer, const LaneBuf& ln, int 
     t.c_idx = ((int)blockIdx.x - cta_off + G) % G;
     t.j0 = min(t.total, t.c_idx * t.q);
     t.j1 = min(t.total, t.j0 + t.q);
+    t.chunk = a.mode == kPrefillChunk;
     t.qkv = ln.qkv;
     t.kv_layer = a.kv + (size_t)layer * a.kv_layer_elems;
-    t.slots = branch ? a.slots + (size_t)layer * a.slot_layer_stride : nullptr;
+    t.slots = (branch && a.mode != kPrefillChunk) ? a.slots + (size_t)layer * a.slot_layer_stride : nullptr;
     t.out = ln.attn; t.partial = ln.partial; t.tickets = ln.tickets;
 }
 
@@ -211,14 +228,17 @@ __device__ void make_phase(const FusedArgs& a, const Prog& P, int ph, int MB, Ph
     phase_info(P, ph, pd.kind, lm, lb);
     pd.n_ops = 0;
     const int G = gridDim.x;
+    const bool chunk = P.mode == kPrefillChunk;
     if (pd.kind == PH_QKV || pd.kind == PH_O || pd.kind == PH_GU || pd.kind == PH_DOWN) {
-        fill_op(a, pd.kind, lm, a.main, 1, 0, pd.op[0]);
+        if (lm >= 0) fill_op(a, pd.kind, lm, a.main, 1, 0, pd.op[0]);
+        else { OpDesc& o = pd.op[0]; o.n_rg = 0; o.n_kc = 0; o.spr = 0; o.first_rg = 0; o.mode = kResid; o.M = 1; o.gain = nullptr; }
         pd.n_ops = 1;
-        if (lb >= 0) { fill_op(a, pd.kind, lb, a.br, MB, G / 2, pd.op[1]); pd.n_ops = 2; }
+        if (lb >= 0) { fill_op(a, pd.kind, lb, a.br, MB, chunk ? 0 : G / 2, pd.op[1]); pd.n_ops = 2; }
     } else if (pd.kind == PH_ATTN) {
-        fill_attn(a, lm, a.main, 1, P.pos, false, 0, pd.at[0]);
+        if (lm >= 0) fill_attn(a, lm, a.main, 1, P.pos, false, 0, pd.at[0]);
+        else { AttnDesc& t = pd.at[0]; t.total = 0; t.j0 = t.j1 = 0; t.q = 1; t.n_splits = 1; t.M = 1; t.chunk = false; }
         pd.n_ops = 1;
-        if (lb >= 0) { fill_attn(a, lb, a.br, MB, P.pos + 1, true, G / 2, pd.at[1]); pd.n_ops = 2; }
+        if (lb >= 0) { fill_attn(a, lb, a.br, MB, chunk ? P.pos : P.pos + 1, true, chunk ? 0 : G / 2, pd.at[1]); pd.n_ops = 2; }
     } else if (pd.kind == PH_HEAD_EARLY || pd.kind == PH_HEAD_FINAL) {
         OpDesc& o = pd.op[0];
         o.w = pd.kind == PH_HEAD_EARLY ? a.w_head_early : a.w_head; o.N = a.V; o.K = a.D; o.x = a.main.h; o.ldx = a.Dp; o.gain = a.g_final; o.resid = nullptr;
@@ -270,7 +290,7 @@ __device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P,
                     it.n_valid = min(kPageTokens, t.p - it.s * kPageTokens);
                     it.tail = it.s == t.s_tail;
                     // a branch row's prefix ends with the position the main pass wrote in this launch
-                    it.kv_late = ln == 1 && it.s == P.pos / kPageTokens;
+                    it.kv_late = P.mode == kPpdStep && ln == 1 && it.s == P.pos / kPageTokens;
                     f(pd, it);
                 }
             }
@@ -696,10 +716,6 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
     const int d0 = lane * DPL;
     const bool lo = d0 < HALF;
     const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
-    float2 cs[DPL];
-#pragma unroll
-    for (int jj = 0; jj < DPL; ++jj) cs[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
-
     for (int jseg = t.j0; jseg < t.j1;) {
         // segment: this CTA's items of one head
         const int h = jseg / t.n_splits;
@@ -741,39 +757,16 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                         const int nv = min(32, n_valid - 32 * hf);              // cached positions in this half
                         const bool has_new = tail && (n_valid >> 5) == hf;     // the new token falls into this half
                         if (nv <= 0 && !has_new) continue;
-                        float qr[DPL], kt[DPL], vt[DPL];
+                        // the row's own position (rows of a prefill chunk sit at consecutive positions)
+                        const int pos_m = t.p + (t.chunk ? m : 0);
+                        float qr[DPL];
 #pragma unroll
                         for (int jj = 0; jj < DPL; ++jj) {
+                            const float2 csq = __ldg(a.rope + (size_t)pos_m * HALF + i0 + jj);
                             const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
-                            qr[jj] = lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]);
-                            kt[jj] = 0.f; vt[jj] = 0.f;
+                            qr[jj] = lo ? rot_lo(x0, x1, csq) : rot_hi(x0, x1, csq);
                         }
-                        if (has_new) {
-                            // the new token: rotate k, round k and v to bf16, store them (branch slot or cache)
-                            const float* kr = qraw + (M + m) * HD;
-                            const float* vr = qraw + (2 * M + m) * HD;
-                            uint16_t kb[DPL], vb[DPL];
-#pragma unroll
-                            for (int jj = 0; jj < DPL; ++jj) {
-                                const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
-                                kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, cs[jj]) : rot_hi(x0, x1, cs[jj]));
-                                vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
-                                kt[jj] = bf16_bits_to_f32(kb[jj]);
-                                vt[jj] = bf16_bits_to_f32(vb[jj]);
-                            }
-                            uint16_t *kd, *vd;
-                            if (t.slots) {
-                                kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
-                                vd = kd + (size_t)H * HD;
-                            } else {
-                                uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
-                                kd = pg + ((size_t)h * kPageTokens + (t.p % kPageTokens)) * HD;
-                                vd = kd + (size_t)H * kPageTokens * HD;
-                            }
-#pragma unroll
-                            for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
-                        }
-                        // scores in log2 units: lane t gets position 32*hf + t; the new token takes lane nv
+                        // scores in log2 units: lane t gets position 32*hf + t; new tokens take lanes nv, nv+1, ..
                         float sc = NEG;
                         if (nv > 0) {
                             float part[32];
@@ -797,18 +790,46 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                             sc = lane < nv ? tot : NEG;
                         }
                         const int nvp = nv > 0 ? nv : 0;
-                        if (has_new) {
+                        // New tokens seen by this row: its own (decode rows), or those of rows 0..m of
+                        // the prefill chunk.  Each is rotated, rounded to bf16 exactly as it is stored;
+                        // the row stores its own.  nvp + n_new <= 32 (the host aligns chunks to 8).
+                        const int n_new = has_new ? (t.chunk ? m + 1 : 1) : 0;
+                        for (int jn = 0; jn < n_new; ++jn) {
+                            const int src = t.chunk ? jn : m;
+                            const int pos_j = t.p + (t.chunk ? jn : 0);
+                            const float* kr = qraw + (M + src) * HD;
+                            const float* vr = qraw + (2 * M + src) * HD;
                             float dsum = 0.f;
+                            uint16_t kb[DPL], vb[DPL];
 #pragma unroll
-                            for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kt[jj], dsum);
+                            for (int jj = 0; jj < DPL; ++jj) {
+                                const float2 csj = __ldg(a.rope + (size_t)pos_j * HALF + i0 + jj);
+                                const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
+                                kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, csj) : rot_hi(x0, x1, csj));
+                                vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
+                                dsum = fmaf(qr[jj], bf16_bits_to_f32(kb[jj]), dsum);
+                            }
+                            if (src == m) {      // store this row's own K/V: branch slot, or the cache at its position
+                                uint16_t *kd, *vd;
+                                if (t.slots) {
+                                    kd = t.slots + (size_t)m * a.slot_stride + (size_t)h * HD;
+                                    vd = kd + (size_t)H * HD;
+                                } else {
+                                    uint16_t* pg = t.kv_layer + (size_t)__ldg(a.page_table + t.s_tail) * page_elems;
+                                    kd = pg + ((size_t)h * kPageTokens + (pos_j % kPageTokens)) * HD;
+                                    vd = kd + (size_t)H * kPageTokens * HD;
+                                }
+#pragma unroll
+                                for (int jj = 0; jj < DPL; ++jj) { kd[d0 + jj] = kb[jj]; vd[d0 + jj] = vb[jj]; }
+                            }
                             dsum = warp_sum(dsum) * sscale;
-                            if (lane == nvp) sc = dsum;        // nvp <= 31: the tail page caches at most 63 positions
+                            if (lane == nvp + jn) sc = dsum;
                         }
-                        const int cnt = nvp + (has_new ? 1 : 0);
+                        const int cnt = nvp + n_new;
                         const float mx = warp_max(sc);
                         const float pr = lane < cnt ? exp2f(sc - mx) : 0.f;
                         const float sum = warp_sum(pr);
-                        // P.V over the cached positions in ascending order, then the new token
+                        // P.V over the cached positions in ascending order, then the new tokens
                         float o[DPL];
 #pragma unroll
                         for (int jj = 0; jj < DPL; ++jj) o[jj] = 0.f;
@@ -824,10 +845,12 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                                 o[0] = fmaf(pw, bf16_lo(vv), o[0]); o[1] = fmaf(pw, bf16_hi(vv), o[1]);
                             }
                         }
-                        if (has_new) {
-                            const float pw = __shfl_sync(0xFFFFFFFFu, pr, nvp);
+                        for (int jn = 0; jn < n_new; ++jn) {
+                            const float pw = __shfl_sync(0xFFFFFFFFu, pr, nvp + jn);
+                            const float* vr = qraw + (2 * M + (t.chunk ? jn : m)) * HD;
 #pragma unroll
-                            for (int jj = 0; jj < DPL; ++jj) o[jj] = fmaf(pw, vt[jj], o[jj]);
+                            for (int jj = 0; jj < DPL; ++jj)
+                                o[jj] = fmaf(pw, bf16_bits_to_f32(f32_to_bf16_bits(vr[d0 + jj])), o[jj]);
                         }
                         // fold this unit into the warp's running state
                         const float nm = fmaxf(run_mx[m], mx);
@@ -981,7 +1004,7 @@ __device__ void state_update(const FusedArgs& a, const Prog& P) {
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
     unsigned long long* base = reinterpret_cast<unsigned long long*>(a.state + S_BAR_BASE);
     *base = *base + (unsigned long long)P.n_phases * gridDim.x;
-    if (P.mode == kPrefillToken) return;
+    if (P.mode == kPrefillToken || P.mode == kPrefillChunk) return;
     const int token = pick_token(a.top_final, a.sample_k, a.temperature, a.sample_u, a.n_sample_u, P.pos);
     int istar = -1;
     if (P.mode == kPpdStep)
@@ -1058,7 +1081,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
                 break;
             case PH_EMBED_BR:
                 if ((int)blockIdx.x < P.k) {
-                    const uint16_t* e = a.emb + (size_t)__ldcg(a.top_early + blockIdx.x) * a.D;
+                    const int tok = P.mode == kPrefillChunk ? __ldcg(a.token_src + blockIdx.x) : __ldcg(a.top_early + blockIdx.x);
+                    const uint16_t* e = a.emb + (size_t)tok * a.D;
                     for (int i = tid; i < a.D; i += kCW * 32) a.br.h[(size_t)blockIdx.x * a.Dp + i] = bf16_bits_to_f32(e[i]);
                 }
                 break;

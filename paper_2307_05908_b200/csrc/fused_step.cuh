@@ -19,7 +19,7 @@ struct LaneBuf {          // activation workspace of one lane (main: 1 row; bran
     int* tickets;         // [H], zero between launches
 };
 
-enum StepMode : int { kPrefillToken = 0, kGreedyStep = 1, kPpdStep = 2 };
+enum StepMode : int { kPrefillToken = 0, kGreedyStep = 1, kPpdStep = 2, kPrefillChunk = 3 };
 
 struct FusedArgs {
     // model
@@ -43,8 +43,8 @@ struct FusedArgs {
     // program
     int mode;              // StepMode
     int k, l;              // PPD: candidates, early layer
-    const int* token_src;  // kPrefillToken: the token to run; otherwise state[S_PENDING] is used
-    int pos_val;           // kPrefillToken: its position
+    const int* token_src;  // kPrefillToken: the token to run; kPrefillChunk: the chunk's k tokens; else state[S_PENDING]
+    int pos_val;           // kPrefillToken / kPrefillChunk: position of the (first) token
     // heads
     float *logits_early, *logits_final;
     int *top_early, *top_final;   // ids[8]; values (float) at +32 words

@@ -84,7 +84,7 @@ Layout plan(const ppd_config& c) {
     L.slot_elems = L.slot_layer_elems * c.n_layers;
     L.slots = take((size_t)(c.max_k > 0 ? c.max_k : 1) * L.slot_elems * 2);
     for (int w = 0; w < 2; ++w) {
-        const size_t rows = c.max_k > 0 ? c.max_k : 1;   // same offsets in both workspaces
+        const size_t rows = kMaxRows;   // a prefill chunk uses up to 8 rows; same offsets in both workspaces
         size_t wo = 0;
         auto wtake = [&](size_t bytes) { size_t r = wo; wo = align_up(wo + bytes, kAlign); return r; };
         L.ws_h = wtake(kMaxRows * (size_t)L.Dp * 4);
@@ -139,6 +139,7 @@ struct ppd_ctx {
     Lane lane[2];
     int* state;
     bool trace;                       // record per-phase timestamps of the fused kernel
+    int prefill_chunk;                // prompt tokens per prefill launch (1, 2, 4 or 8)
     int sample_k, n_sample_u;         // top-k sampling of the final prediction (0 = greedy)
     float temperature;
     const uint16_t* w_early;          // packed classifier of the early head in caller memory, or nullptr = W_H
@@ -446,14 +447,20 @@ int decode_fused(ppd_ctx* x, int k, int l, int n, int eos, int32_t* out_tokens, 
     return PPD_OK;
 }
 
+// Prompt positions 0..n_prompt-2 in chunks of consecutive tokens (4 by default, at most 8): one launch per chunk, the
+// chunk's tokens are the rows of one weight pass and attend causally to each other.  Chunks start at
+// multiples of 8, so a chunk never straddles a KV page or a 32-position half page.
 int prefill_fused(ppd_ctx* x, int n_prompt) {
     FusedArgs f;
     fill_fused(x, f);
-    f.mode = kPrefillToken;
-    for (int t = 0; t + 1 < n_prompt; ++t) {
-        f.token_src = at<int>(x, x->L.prompt) + t;
-        f.pos_val = t;
-        CK(launch_fused_step(f, 0, x->sm, x->pdl, x->n_sms));
+    const int chunk = x->prefill_chunk;
+    f.mode = chunk == 1 ? kPrefillToken : kPrefillChunk;     // one token at a time runs on the main lane
+    for (int t0 = 0; t0 + 1 < n_prompt; t0 += chunk) {
+        const int m = n_prompt - 1 - t0 < chunk ? n_prompt - 1 - t0 : chunk;
+        f.k = m;
+        f.token_src = at<int>(x, x->L.prompt) + t0;
+        f.pos_val = t0;
+        CK(launch_fused_step(f, chunk == 1 ? 0 : m, x->sm, x->pdl, x->n_sms));
     }
     return PPD_OK;
 }
@@ -503,6 +510,7 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     x->pdl = true;
     x->fused = true;
     x->w_early = nullptr;
+    x->prefill_chunk = 4;
     x->sample_k = 0; x->n_sample_u = 0; x->temperature = 1.f;
     x->trace = false;
     x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
@@ -640,6 +648,12 @@ int ppd_load_early_head(ppd_ctx* x, const void* host_w, size_t bytes, int dtype,
     }
     CK(cudaStreamSynchronize(x->sm));
     x->w_early = dst;
+    return PPD_OK;
+}
+
+int ppd_set_prefill_chunk(ppd_ctx* x, int32_t n_tokens) {
+    if (!x || (n_tokens != 1 && n_tokens != 2 && n_tokens != 4 && n_tokens != 8)) return PPD_EINVAL;
+    x->prefill_chunk = n_tokens;
     return PPD_OK;
 }
 

@@ -312,6 +312,33 @@ def test_sampled_final_prediction(tiny_ctx, tiny_shape, tiny_blob, tiny_prompt):
         tiny_ctx.set_sampling(0)
 
 
+def test_prefill_chunk_sizes_agree(tiny_shape, tiny_blob):
+    """Chunked prefill (several prompt tokens per weight pass, causal inside the chunk) against
+    token-by-token prefill: same cache up to rounding, and PPD == greedy after either."""
+    prompt = ppd_inputs.gen_prompt(tiny_shape.vocab, 203, seed=21)       # ragged last chunk, several pages
+    ctx = ppd.Context(tiny_shape, max_seq=260, max_k=3)
+    ctx.load_weights(tiny_blob)
+    ref = None
+    for chunk in (1, 2, 4, 8):
+        ctx.set_prefill_chunk(chunk)
+        ctx.prefill(prompt)
+        t, h = ctx.step(3, 2)
+        lg = ctx.debug_logits()
+        ctx.prefill(prompt)
+        g, _ = ctx.decode(0, 0, 20)
+        ctx.prefill(prompt)
+        p, _ = ctx.decode(3, 2, 20)
+        assert (p == g).all()
+        if ref is None:
+            ref = lg
+        assert np.abs(lg - ref).max() < 1e-4
+    o = Oracle(tiny_shape, tiny_blob, max_seq=260)
+    o.prefill(prompt)
+    r = o.greedy_probe(1, dump_logits=True)
+    assert np.abs(lg - r["final_logits"][0]).max() < 1e-3
+    ctx.close()
+
+
 def test_modes_agree_and_can_be_switched(tiny_shape, tiny_blob, tiny_prompt):
     ctx = ppd.Context(tiny_shape, max_seq=96, max_k=5)
     ctx.load_weights(tiny_blob)
