@@ -480,22 +480,30 @@ __device__ __forceinline__ void select8(const float* vals, const int* ids, int n
 }
 
 // One matrix product: this CTA's row groups, stages taken from the ring in program order.
+//
+// Work split inside a 32-row x 256-column tile: warp w takes the 64-column slice (w & 3) of the row
+// half (w >> 2); lane l takes the 8 columns (l & 7) of that slice for the rows (l >> 3) + 4 i, i < 4,
+// of the half.  A quarter warp therefore reads 128 contiguous bytes of one tile row (no bank
+// conflicts with the plain row-major tile), and an activation slice is read by two warps instead of
+// eight -- with several batch rows the activations, not the weights, dominate shared-memory traffic.
+// Per (batch row, weight row) the order of additions is fixed: a lane's column pairs tile after
+// tile into one packed {even, odd} accumulator, the two halves, a shuffle tree over the 8 lanes of a
+// slice, then the four slices in order through shared memory.
 // RMSNorm is applied as  y = (sum_k W[n][k] * (g[k] h[k])) / rms(h): the sum of squares is
 // gathered from the same slices while the first row group streams by, so no extra pass over h.
 template <int M, int MODE, bool NORM, int MB>
-__device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, float* lv, int* li) {
+__device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb, float* lv, int* li) {
     using C = Cfg<MB>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x;
     int* err = a.state + S_ERR;
-    const int r0 = warp * 4;
-    // Per (row of the batch, weight row): one packed accumulator {sum over even k, sum over odd k};
-    // a lane adds its four column pairs of every tile in a fixed order, the halves are added at the
-    // end, then the lanes are summed by a fixed shuffle tree.
-    float inv[M];
+    const int sl = warp & 3, hf = warp >> 2, c8 = lane & 7, rq = lane >> 3;
+    const int w_off = (hf * 16 + rq) * 32 + sl * 8 + c8;          // uint4 index of (first row, column chunk) in a tile
+    const int x_off = sl * 16 + c8 * 2;                           // ulonglong2 index of the lane's 8 activations in a tile's slice
     unsigned long long ssq[M];
 #pragma unroll
-    for (int m = 0; m < M; ++m) { inv[m] = 1.f; ssq[m] = 0ull; }
+    for (int m = 0; m < M; ++m) ssq[m] = 0ull;
+    float inv = 1.f;                                              // of batch row (tid >> 5); used by the epilogue threads
     bool first = true;
     for (int rg = op.first_rg; rg < op.n_rg; rg += G) {
         unsigned long long acc2[M][4];
@@ -511,20 +519,20 @@ __device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared&
 #pragma unroll
             for (int t = 0; t < kTS; ++t) {
                 if (t < nt) {
-                    const uint4* wt = reinterpret_cast<const uint4*>(st + t * kTileBytes) + r0 * 32 + lane;
+                    const uint4* wt = reinterpret_cast<const uint4*>(st + t * kTileBytes) + w_off;
                     uint4 w[4];
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) w[r] = wt[r * 32];
+                    for (int r = 0; r < 4; ++r) w[r] = wt[r * 4 * 32];
                     unsigned long long xv[M][4];
                     unsigned long long gs[4];
                     if (NORM) {
-                        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(st + C::kGOff) + t * (kTileCols / 4) + lane * 2;
+                        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(st + C::kGOff) + t * (kTileCols / 4) + x_off;
                         const ulonglong2 g0 = gp[0], g1 = gp[1];
                         gs[0] = g0.x; gs[1] = g0.y; gs[2] = g1.x; gs[3] = g1.y;
                     }
 #pragma unroll
                     for (int m = 0; m < M; ++m) {
-                        const ulonglong2* xp = reinterpret_cast<const ulonglong2*>(st + C::kXOff + m * kRowX) + t * (kTileCols / 4) + lane * 2;
+                        const ulonglong2* xp = reinterpret_cast<const ulonglong2*>(st + C::kXOff + m * kRowX) + t * (kTileCols / 4) + x_off;
                         const ulonglong2 x0 = xp[0], x1 = xp[1];
                         xv[m][0] = x0.x; xv[m][1] = x0.y; xv[m][2] = x1.x; xv[m][3] = x1.y;
                         if (NORM) {
@@ -551,81 +559,87 @@ __device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared&
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
         }
-        if (NORM && first) {
+        // partial sums of the slice -> shared memory: red[slice][batch row][tile row], then ssq[slice][batch row]
+        float* red = reinterpret_cast<float*>(sh.un) + rb * (4 * C::MR * 33);
+        float* red_q = red + 4 * C::MR * 32;
 #pragma unroll
-            for (int m = 0; m < M; ++m) {
-                float s0, s1;
-                unpack2(ssq[m], s0, s1);
-                inv[m] = 1.0f / sqrtf(warp_sum(s0 + s1) / (float)op.K + a.eps);
-            }
-        }
-        first = false;
-        float acc[M][4];
-#pragma unroll
-        for (int m = 0; m < M; ++m)
+        for (int m = 0; m < M; ++m) {
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 float s0, s1;
                 unpack2(acc2[m][r], s0, s1);
-                acc[m][r] = warp_sum(s0 + s1);
-                if (NORM) acc[m][r] = __fmul_rn(acc[m][r], inv[m]);
+                float v = s0 + s1;
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+                if (c8 == 0) red[(sl * C::MR + m) * 32 + hf * 16 + rq + 4 * r] = v;
             }
-        const int n0 = rg * kTileRows + r0;
-        if (MODE == kStore || MODE == kResid || MODE == kHead) {
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                const float v = lane == 0 ? acc[m][0] : lane == 1 ? acc[m][1] : lane == 2 ? acc[m][2] : acc[m][3];
-                const int n = n0 + lane;
-                if (lane < 4 && n < op.N) {
+            if (NORM && first) {
+                float s0, s1;
+                unpack2(ssq[m], s0, s1);
+                float v = s0 + s1;
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+                if (hf == 0 && lane == 0) red_q[sl * C::MR + m] = v;
+            }
+        }
+        consumer_sync();
+        rb ^= 1;      // the next row group writes the other buffer while the epilogue threads read this one
+        if (warp < M) {      // warp m finishes batch row m: lane = row of the tile
+            const int m = warp;
+            if (NORM && first)
+                inv = 1.0f / sqrtf((((red_q[m] + red_q[C::MR + m]) + red_q[2 * C::MR + m]) + red_q[3 * C::MR + m]) / (float)op.K + a.eps);
+            float v = ((red[m * 32 + lane] + red[(C::MR + m) * 32 + lane]) + red[(2 * C::MR + m) * 32 + lane]) + red[(3 * C::MR + m) * 32 + lane];
+            if (NORM) v = __fmul_rn(v, inv);
+            const int n = rg * kTileRows + lane;
+            if (MODE == kSwiglu) {
+                const float u = __shfl_down_sync(0xFFFFFFFFu, v, 1);
+                if (!(lane & 1) && n + 1 < op.N) op.out[(size_t)m * op.ldo + (n >> 1)] = (v / (1.0f + expf(-v))) * u;
+            } else {
+                if (n < op.N) {
                     const size_t o = (size_t)m * op.ldo + n;
                     op.out[o] = (MODE == kResid) ? __ldcg(op.resid + o) + v : v;
                 }
                 if (MODE == kHead) {
-#pragma unroll
-                    for (int r = 0; r < 4; ++r)
-                        if (n0 + r < op.N) list_insert(lv[m], li[m], acc[m][r], n0 + r, lane);
+                    // only values that beat the current 8th best enter the ordered list
+                    const float v8 = __shfl_sync(0xFFFFFFFFu, lv[0], 7);
+                    const int i8 = __shfl_sync(0xFFFFFFFFu, li[0], 7);
+                    unsigned cand = __ballot_sync(0xFFFFFFFFu, n < op.N && better(v, n, v8, i8));
+                    while (cand) {
+                        const int src = __ffs(cand) - 1;
+                        cand &= cand - 1;
+                        list_insert(lv[0], li[0], __shfl_sync(0xFFFFFFFFu, v, src), rg * kTileRows + src, lane);
+                    }
                 }
             }
-        } else {
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                const float g = lane == 0 ? acc[m][0] : acc[m][2];
-                const float u = lane == 0 ? acc[m][1] : acc[m][3];
-                const int j = (n0 >> 1) + lane;
-                if (lane < 2 && 2 * j + 1 < op.N) op.out[(size_t)m * op.ldo + j] = (g / (1.0f + expf(-g))) * u;
-            }
         }
+        first = false;
     }
 }
 
 template <int M, int MB>
-__device__ void run_gemv_op(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it) {
+__device__ void run_gemv_op(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb) {
     float lv[1]; int li[1];
     switch (op.mode) {
-        case kStore: gemv_consume<M, kStore, true, MB>(a, op, sh, it, lv, li); break;
-        case kSwiglu: gemv_consume<M, kSwiglu, true, MB>(a, op, sh, it, lv, li); break;
-        default: gemv_consume<M, kResid, false, MB>(a, op, sh, it, lv, li); break;
+        case kStore: gemv_consume<M, kStore, true, MB>(a, op, sh, it, rb, lv, li); break;
+        case kSwiglu: gemv_consume<M, kSwiglu, true, MB>(a, op, sh, it, rb, lv, li); break;
+        default: gemv_consume<M, kResid, false, MB>(a, op, sh, it, rb, lv, li); break;
     }
 }
 
-// Head (one row): logits + top-8.  Per-warp lists -> CTA list -> global lists -> the last CTA to
-// arrive merges them (atomic ticket; nobody waits).
+// Head (one row): logits + top-8.  Warp 0 keeps the CTA's ordered list -> global lists -> the last
+// CTA to arrive merges them (atomic ticket; nobody waits).
 template <int MB>
-__device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int* top_out) {
+__device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb, int* top_out) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     float lv[1] = {__int_as_float(0xFF800000)};
     int li[1] = {0x7FFFFFFF};
-    gemv_consume<1, kHead, true, MB>(a, op, sh, it, lv, li);
-    if (lane < 8) { sh.lists_v[warp * 8 + lane] = lv[0]; sh.lists_i[warp * 8 + lane] = li[0]; }
-    consumer_sync();
+    gemv_consume<1, kHead, true, MB>(a, op, sh, it, rb, lv, li);
     int* ticket = a.state + S_HEAD_TICKET;
     float* gv = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.head_scratch) + 256);
     int* gi = reinterpret_cast<int*>(gv + (size_t)kMaxRows * kHeadMaxCtas * 8);
-    if (warp == 0) {
-        float ov; int oi;
-        select8(sh.lists_v, sh.lists_i, kCW * 8, lane, ov, oi);
-        if (lane < 8) { gv[blockIdx.x * 8 + lane] = ov; gi[blockIdx.x * 8 + lane] = oi; }
-    }
+    if (warp == 0 && lane < 8) { gv[blockIdx.x * 8 + lane] = lv[0]; gi[blockIdx.x * 8 + lane] = li[0]; }
     __threadfence();
     consumer_sync();
     if (tid == 0) sh.flags[0] = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
@@ -716,6 +730,12 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
     const int d0 = lane * DPL;
     const bool lo = d0 < HALF;
     const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
+    // rotation of position p (every decode row sits there), fetched before the first stage arrives
+    float2 cs_p[DPL];
+    if (t.j0 < t.j1) {
+#pragma unroll
+        for (int jj = 0; jj < DPL; ++jj) cs_p[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
+    }
     for (int jseg = t.j0; jseg < t.j1;) {
         // segment: this CTA's items of one head
         const int h = jseg / t.n_splits;
@@ -762,7 +782,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                         float qr[DPL];
 #pragma unroll
                         for (int jj = 0; jj < DPL; ++jj) {
-                            const float2 csq = __ldg(a.rope + (size_t)pos_m * HALF + i0 + jj);
+                            const float2 csq = t.chunk ? __ldg(a.rope + (size_t)pos_m * HALF + i0 + jj) : cs_p[jj];
                             const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
                             qr[jj] = lo ? rot_lo(x0, x1, csq) : rot_hi(x0, x1, csq);
                         }
@@ -803,7 +823,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                             uint16_t kb[DPL], vb[DPL];
 #pragma unroll
                             for (int jj = 0; jj < DPL; ++jj) {
-                                const float2 csj = __ldg(a.rope + (size_t)pos_j * HALF + i0 + jj);
+                                const float2 csj = t.chunk ? __ldg(a.rope + (size_t)pos_j * HALF + i0 + jj) : cs_p[jj];
                                 const float x0 = kr[i0 + jj], x1 = kr[i0 + jj + HALF];
                                 kb[jj] = f32_to_bf16_bits(lo ? rot_lo(x0, x1, csj) : rot_hi(x0, x1, csj));
                                 vb[jj] = f32_to_bf16_bits(vr[d0 + jj]);
@@ -1063,7 +1083,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
 
     int* err = a.state + S_ERR;
     unsigned long long* cnt = reinterpret_cast<unsigned long long*>(a.state + S_BAR_COUNT);
-    int it = 0;
+    int it = 0, rb = 0;
     PhaseDesc pd;
     for (int ph = 0; ph < P.n_phases; ++ph) {
         make_phase(a, P, ph, MB, pd);        // overlaps the barrier latency
@@ -1087,8 +1107,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
                 }
                 break;
             case PH_QKV: case PH_O: case PH_GU: case PH_DOWN:
-                run_gemv_op<1, MB>(a, pd.op[0], sh, it);
-                if (MB > 0 && pd.n_ops == 2) run_gemv_op<(MB > 0 ? MB : 1), MB>(a, pd.op[1], sh, it);
+                run_gemv_op<1, MB>(a, pd.op[0], sh, it, rb);
+                if (MB > 0 && pd.n_ops == 2) run_gemv_op<(MB > 0 ? MB : 1), MB>(a, pd.op[1], sh, it, rb);
                 break;
             case PH_ATTN:
                 run_attn<1, MB>(a, pd.at[0], sh, it);
@@ -1099,10 +1119,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
                 if (MB > 0 && pd.n_ops == 2) run_attn_merge<(MB > 0 ? MB : 1), MB>(a, pd.at[1], sh);
                 break;
             case PH_HEAD_EARLY:
-                run_head<MB>(a, pd.op[0], sh, it, a.top_early);
+                run_head<MB>(a, pd.op[0], sh, it, rb, a.top_early);
                 break;
             case PH_HEAD_FINAL:
-                run_head<MB>(a, pd.op[0], sh, it, a.top_final);
+                run_head<MB>(a, pd.op[0], sh, it, rb, a.top_final);
                 break;
             case PH_COMMIT:
                 commit_copy(a, P);
