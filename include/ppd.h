@@ -109,9 +109,14 @@ int ppd_set_sampling(ppd_ctx* ctx, int32_t top_k, float temperature, const float
  * mode the prompt runs through the step kernel in chunks of 4 tokens per launch. */
 int ppd_prefill(ppd_ctx* ctx, const int32_t* prompt, int32_t n_prompt);
 
-/* Prompt tokens processed per prefill launch in the default mode: 4 (default), 8, 2 or 1.  The
- * tokens of a chunk share one pass over the weights and attend causally to each other; chunk
- * sizes differ in rounding only. */
+/* How ppd_prefill processes the prompt.
+ *   n_tokens = 4 (default), 8, 2 or 1: through the step kernel, that many prompt tokens per launch;
+ *     the tokens of a chunk share one pass over the weights and attend causally to each other.
+ *   n_tokens = 0: on the tensor cores -- the prompt rows (up to 1024 per pass) go through tcgen05
+ *     matrix products (activations as bf16 hi + lo pairs, fp32 accumulation) and a causal
+ *     attention kernel over the paged cache.  The paper only says that the prompt is forwarded
+ *     ("x<=t" in Algorithm 1); this is the one dense contraction of the method.
+ * All settings differ in float rounding only. */
 int ppd_set_prefill_chunk(ppd_ctx* ctx, int32_t n_tokens);
 
 /* One conventional greedy step: all d layers, argmax of the final logits (Section 1).
@@ -203,6 +208,15 @@ int ppd_op_pack(const uint16_t* src, int32_t n_src_rows, int32_t n_cols, void* d
 int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
                 const float* gain, float eps, int32_t mode, const float* resid, float* out,
                 int32_t ldo, void* stream);
+
+/* Many-row matrix product on the tensor cores (the prompt path's building block):
+ * out[m][n] = sum_k W[n][k] x[m][k] for m < M (any M >= 1), fp32 accumulation, x split into bf16
+ * hi + lo pairs.  w_packed: device, packed [N][K].  x: device float32 [M][ldx].  out: device
+ * float32 [M][ldo].  scratch: device, >= ppd_op_gemm_scratch_bytes(M, K) bytes, 256-byte aligned.
+ * Synchronises the stream; PPD_ETIMEOUT if a bounded device wait gave up. */
+size_t ppd_op_gemm_scratch_bytes(int32_t M, int32_t K);
+int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
+                float* out, int32_t ldo, void* scratch, size_t scratch_bytes, void* stream);
 
 /* Head: logits[m][v] = W_H . RMSNorm(x[m]) for M rows and the k largest per row in the order
  * (value descending, id ascending).  scratch: device, >= ppd_op_head_scratch_bytes() bytes,

@@ -69,6 +69,8 @@ SIGNATURES = {
     "ppd_packed_bytes": (_SZ, [_I, _I]),
     "ppd_op_pack": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _I, _P]),
     "ppd_op_gemv": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _I, _P]),
+    "ppd_op_gemm_scratch_bytes": (_SZ, [_I, _I]),
+    "ppd_op_gemm": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _I, _P, _SZ, _P]),
     "ppd_op_head_scratch_bytes": (_SZ, []),
     "ppd_op_head_topk": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P, _P]),
     "ppd_op_head_topk_static": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P]),
@@ -291,6 +293,17 @@ def op_gemv(w_packed, N, K, x, gain, eps, mode, resid, out, stream=None):
     _check(load().ppd_op_gemv(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx,
                               None if gain is None else gain.data_ptr(), eps, mode,
                               None if resid is None else resid.data_ptr(), out.data_ptr(), out.shape[1], _s(stream)))
+
+
+def op_gemm_scratch_bytes(M, K):
+    return load().ppd_op_gemm_scratch_bytes(M, K)
+
+
+def op_gemm(w_packed, N, K, x, out, scratch, stream=None):
+    """out[m][n] = sum_k W[n][k] x[m][k] on the tensor cores; x, out float32 device tensors."""
+    M, ldx = x.shape
+    _check(load().ppd_op_gemm(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx, out.data_ptr(), out.shape[1],
+                              scratch.data_ptr(), scratch.numel() * scratch.element_size(), _s(stream)))
 
 
 def op_head_topk(w_packed, vocab, K, x, gain, eps, k, scratch, logits, top_ids, top_vals, stream=None):

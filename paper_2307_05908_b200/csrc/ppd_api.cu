@@ -11,6 +11,7 @@
 #include "../../include/ppd.h"
 #include "common.cuh"
 #include "fused_step.cuh"
+#include "prefill_tc.cuh"
 #include "gemv.cuh"
 #include "misc.cuh"
 
@@ -21,6 +22,7 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr size_t kStagingBytes = 64ull << 20;
 constexpr int kTimelinePhases = 512;
+constexpr int kPfMaxRows = 1024;     // prompt rows per pass of the tensor-core path
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int round_up(int v, int a) { return (v + a - 1) / a * a; }
@@ -36,6 +38,8 @@ struct Layout {
     size_t ws_h, ws_qkv, ws_attn, ws_z, ws_part, ws_tick, ws_bytes[2];   // offsets inside a workspace
     size_t logits_final, logits_early, top_final, top_early, head_scratch;
     size_t state, sample_u, prompt, out_tokens, out_hit, out_margin, timeline, staging, total;
+    size_t pf_h, pf_qkv, pf_xhi, pf_xlo, pf_zhi, pf_zlo;   // tensor-core prompt path: activations of up to pf_rows tokens
+    int pf_rows;
 };
 
 bool valid_config(const ppd_config* c) {
@@ -111,6 +115,16 @@ Layout plan(const ppd_config& c) {
     L.out_margin = take((size_t)c.max_seq * 4);
     L.timeline = take(kTimelinePhases * 2 * 2 * 8);
     L.staging = take(kStagingBytes);
+    {
+        const int want = (c.max_seq + kTcBM - 1) / kTcBM * kTcBM;
+        L.pf_rows = want < kPfMaxRows ? want : kPfMaxRows;
+        L.pf_h = take((size_t)L.pf_rows * L.Dp * 4);
+        L.pf_qkv = take((size_t)L.pf_rows * 3 * D * 4);
+        L.pf_xhi = take((size_t)L.pf_rows * L.Dp * 2);
+        L.pf_xlo = take((size_t)L.pf_rows * L.Dp * 2);
+        L.pf_zhi = take((size_t)L.pf_rows * L.Fp * 2);
+        L.pf_zlo = take((size_t)L.pf_rows * L.Fp * 2);
+    }
     L.total = o;
     return L;
 }
@@ -139,7 +153,10 @@ struct ppd_ctx {
     Lane lane[2];
     int* state;
     bool trace;                       // record per-phase timestamps of the fused kernel
-    int prefill_chunk;                // prompt tokens per prefill launch (1, 2, 4 or 8)
+    int prefill_chunk;                // prompt tokens per prefill launch (1, 2, 4 or 8); 0 = tensor-core path
+    bool tc_ok;                       // tensor maps of the tensor-core prompt path are ready
+    CUtensorMap map_xhi, map_xlo, map_zhi, map_zlo;
+    std::vector<CUtensorMap> map_w;   // per layer: Wqkv, Wo, Wgu, Wd
     int sample_k, n_sample_u;         // top-k sampling of the final prediction (0 = greedy)
     float temperature;
     const uint16_t* w_early;          // packed classifier of the early head in caller memory, or nullptr = W_H
@@ -465,6 +482,52 @@ int prefill_fused(ppd_ctx* x, int n_prompt) {
     return PPD_OK;
 }
 
+// Prompt positions 0..n_prompt-2 on the tensor cores, up to pf_rows tokens per pass: every matrix
+// product of a decoder block is one tcgen05 GEMM over the pass's rows; the rows' K/V go to the cache
+// before the causal attention kernel reads it.
+int prefill_tc(ppd_ctx* x, int n_prompt) {
+    if (!x->tc_ok) return PPD_ECUDA;
+    const ppd_config& c = x->c;
+    const Layout& L = x->L;
+    const int D = c.d_model, F = c.d_ffn;
+    float* h = at<float>(x, L.pf_h);
+    float* qkv = at<float>(x, L.pf_qkv);
+    uint16_t *xhi = at<uint16_t>(x, L.pf_xhi), *xlo = at<uint16_t>(x, L.pf_xlo);
+    uint16_t *zhi = at<uint16_t>(x, L.pf_zhi), *zlo = at<uint16_t>(x, L.pf_zlo);
+    for (int t0 = 0; t0 + 1 < n_prompt; t0 += L.pf_rows) {
+        const int m = n_prompt - 1 - t0 < L.pf_rows ? n_prompt - 1 - t0 : L.pf_rows;
+        CK(launch_pf_embed(at<uint16_t>(x, L.emb), at<int>(x, L.prompt) + t0, m, D, h, L.Dp, x->sm));
+        for (int l = 0; l < c.n_layers; ++l) {
+            uint8_t* lb = layer_block(x, l);
+            const CUtensorMap* mw = &x->map_w[(size_t)l * 4];
+            TcGemmArgs g{};
+            g.m_rows = m;
+            g.err = x->state + S_ERR;
+            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g1), c.rms_eps, m, D, xhi, xlo, L.Dp, x->sm));
+            g.n_cols = 3 * D; g.k_blocks = (D + kTcBK - 1) / kTcBK; g.mode = kTcStore; g.out = qkv; g.ldo = 3 * D;
+            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[0], g, x->sm));
+            PfKvArgs kv{};
+            kv.qkv = qkv; kv.rows = m; kv.H = c.n_heads; kv.hd = c.head_dim; kv.D = D; kv.pos0 = t0;
+            kv.rope = at<float2>(x, L.rope);
+            kv.kv_layer = at<uint16_t>(x, L.kv) + (size_t)l * L.kv_layer_elems;
+            kv.page_table = at<int>(x, L.page_table);
+            CK(launch_pf_rope_kv(kv, x->sm));
+            PfAttnArgs pa{};
+            pa.qkv = qkv; pa.rows = m; pa.H = c.n_heads; pa.hd = c.head_dim; pa.D = D; pa.pos0 = t0;
+            pa.kv_layer = kv.kv_layer; pa.page_table = kv.page_table; pa.out_hi = xhi; pa.out_lo = xlo; pa.ld = L.Dp;
+            CK(launch_pf_attn(pa, x->sm));
+            g.n_cols = D; g.mode = kTcResid; g.out = h; g.ldo = L.Dp;
+            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[1], g, x->sm));
+            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g2), c.rms_eps, m, D, xhi, xlo, L.Dp, x->sm));
+            g.n_cols = 2 * F; g.mode = kTcSwigluSplit; g.out = nullptr; g.out_hi = zhi; g.out_lo = zlo; g.ld_hl = L.Fp;
+            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[2], g, x->sm));
+            g.n_cols = D; g.k_blocks = (F + kTcBK - 1) / kTcBK; g.mode = kTcResid; g.out = h; g.ldo = L.Dp;
+            CK(launch_tc_gemm(x->map_zhi, x->map_zlo, mw[3], g, x->sm));
+        }
+    }
+    return PPD_OK;
+}
+
 int check_decode_args(ppd_ctx* x, int k, int l, int n) {
     if (!x) return PPD_EINVAL;
     if (!x->loaded || !x->prefilled) return PPD_ESTATE;
@@ -547,6 +610,24 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
         x->lane[w].z = reinterpret_cast<float*>(ws + L.ws_z);
         x->lane[w].partial = reinterpret_cast<float*>(ws + L.ws_part);
         x->lane[w].tickets = reinterpret_cast<int*>(ws + L.ws_tick);
+    }
+    // tensor maps of the tensor-core prompt path (device addresses only; nothing is read here)
+    x->tc_ok = tc_init() == 0;
+    if (x->tc_ok) {
+        const int D = cfg->d_model, F = cfg->d_ffn;
+        x->tc_ok = tc_map_rows(&x->map_xhi, at<uint16_t>(x, L.pf_xhi), L.pf_rows, L.Dp) == 0 &&
+                   tc_map_rows(&x->map_xlo, at<uint16_t>(x, L.pf_xlo), L.pf_rows, L.Dp) == 0 &&
+                   tc_map_rows(&x->map_zhi, at<uint16_t>(x, L.pf_zhi), L.pf_rows, L.Fp) == 0 &&
+                   tc_map_rows(&x->map_zlo, at<uint16_t>(x, L.pf_zlo), L.pf_rows, L.Fp) == 0;
+        x->map_w.resize((size_t)cfg->n_layers * 4);
+        for (int l = 0; l < cfg->n_layers && x->tc_ok; ++l) {
+            uint8_t* lb = layer_block(x, l);
+            CUtensorMap* mw = &x->map_w[(size_t)l * 4];
+            x->tc_ok = tc_map_packed(&mw[0], reinterpret_cast<uint16_t*>(lb + L.off_wqkv), 3 * D, D) == 0 &&
+                       tc_map_packed(&mw[1], reinterpret_cast<uint16_t*>(lb + L.off_wo), D, D) == 0 &&
+                       tc_map_packed(&mw[2], reinterpret_cast<uint16_t*>(lb + L.off_wgu), 2 * F, D) == 0 &&
+                       tc_map_packed(&mw[3], reinterpret_cast<uint16_t*>(lb + L.off_wd), D, F) == 0;
+        }
     }
     *out = x;
     return PPD_OK;
@@ -652,7 +733,8 @@ int ppd_load_early_head(ppd_ctx* x, const void* host_w, size_t bytes, int dtype,
 }
 
 int ppd_set_prefill_chunk(ppd_ctx* x, int32_t n_tokens) {
-    if (!x || (n_tokens != 1 && n_tokens != 2 && n_tokens != 4 && n_tokens != 8)) return PPD_EINVAL;
+    if (!x || (n_tokens != 0 && n_tokens != 1 && n_tokens != 2 && n_tokens != 4 && n_tokens != 8)) return PPD_EINVAL;
+    if (n_tokens == 0 && !x->tc_ok) return PPD_ECUDA;
     x->prefill_chunk = n_tokens;
     return PPD_OK;
 }
@@ -684,7 +766,10 @@ int ppd_prefill(ppd_ctx* x, const int32_t* prompt, int32_t n_prompt) {
     CK(cudaMemcpyAsync(x->base + L.prompt, prompt, (size_t)n_prompt * 4, cudaMemcpyHostToDevice, x->sm));
     CK(cudaStreamSynchronize(x->sm));   // the host array may be reused by the caller
     const int64_t launches = x->stats.kernel_launches;
-    if (x->fused) {
+    if (x->prefill_chunk == 0) {
+        int rc = prefill_tc(x, n_prompt);
+        if (rc) return rc;
+    } else if (x->fused) {
         int rc = prefill_fused(x, n_prompt);
         if (rc) return rc;
     } else {
@@ -906,6 +991,37 @@ int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int3
     g.resid = resid; g.out = out; g.ldo = ldo; g.err = nullptr;
     CKOP(launch_gemv(g, M, mode, reinterpret_cast<cudaStream_t>(stream), false, sm_count()));
     return PPD_OK;
+}
+
+size_t ppd_op_gemm_scratch_bytes(int32_t M, int32_t K) {
+    if (M < 1 || K < 1) return 0;
+    return (size_t)2 * round_up(M, kTcBM) * round_up(K, kTileCols) * 2 + 256;
+}
+
+int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, float* out,
+                int32_t ldo, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!w_packed || !x || !out || !scratch || N < 1 || K < 1 || M < 1 || ldx < K || ldo < N) return PPD_EINVAL;
+    if (((uintptr_t)scratch % kAlign) != 0) return PPD_EINVAL;
+    if (scratch_bytes < ppd_op_gemm_scratch_bytes(M, K)) return PPD_ENOSPC;
+    if (tc_init() != 0) return PPD_ECUDA;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int Mp = (int)round_up(M, kTcBM), Kp = (int)round_up(K, kTileCols);
+    int* err = reinterpret_cast<int*>(scratch);
+    uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256);
+    uint16_t* lo = hi + (size_t)Mp * Kp;
+    CKOP(cudaMemsetAsync(scratch, 0, ppd_op_gemm_scratch_bytes(M, K), st));
+    CKOP(launch_pf_norm_split(x, ldx, nullptr, 0.f, M, K, hi, lo, Kp, st));
+    CUtensorMap ma, mb, mw;
+    if (tc_map_rows(&ma, hi, Mp, Kp) || tc_map_rows(&mb, lo, Mp, Kp) ||
+        tc_map_packed(&mw, reinterpret_cast<const uint16_t*>(w_packed), N, K))
+        return PPD_ECUDA;
+    TcGemmArgs g{};
+    g.m_rows = M; g.n_cols = N; g.k_blocks = (K + kTcBK - 1) / kTcBK; g.mode = kTcStore; g.out = out; g.ldo = ldo; g.err = err;
+    CKOP(launch_tc_gemm(ma, mb, mw, g, st));
+    int h_err = 0;
+    CKOP(cudaMemcpyAsync(&h_err, err, 4, cudaMemcpyDeviceToHost, st));
+    CKOP(cudaStreamSynchronize(st));
+    return h_err ? PPD_ETIMEOUT : PPD_OK;
 }
 
 size_t ppd_op_head_scratch_bytes(void) { return kHeadScratchBytes + 2 * kMaxRows * 8 * 4; }

@@ -1,0 +1,440 @@
+// Prompt processing on the tensor cores: tcgen05 matrix products with the accumulator in tensor
+// memory, operands staged by TMA tensor copies, plus the small kernels around them (embedding rows,
+// RMSNorm + bf16 hi/lo split, rotary embedding + KV write, causal attention over the paged cache).
+//
+// Precision: the weights are bf16 already; an activation x (fp32) enters the tensor cores as the
+// pair hi = bf16(x), lo = bf16(x - hi), two matrix instructions per tile, so x is represented to
+// about 2^-17 relative and the products are exact in the fp32 accumulator.  This keeps the prompt's
+// K/V and hidden states within float rounding of the decode path's.
+#include "common.cuh"
+#include "prefill_tc.cuh"
+
+namespace ppd {
+namespace {
+
+// ------------------------------------------------------------------------------------------ host: tensor maps
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+}  // namespace
+
+int tc_init() {
+    if (g_encode) return 0;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess) return -1;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return -1;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return 0;
+}
+
+int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols) {
+    if (!g_encode || cols % kTcBK != 0) return -1;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)kTcBM};
+    const cuuint32_t es[2] = {1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(base), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+               ? 0
+               : -1;
+}
+
+int tc_map_packed(CUtensorMap* map, const uint16_t* packed, int n_rows, int n_cols) {
+    if (!g_encode) return -1;
+    const cuuint64_t n_rg = (n_rows + kTileRows - 1) / kTileRows, n_kc = (n_cols + kTileCols - 1) / kTileCols;
+    const cuuint64_t dims[4] = {(cuuint64_t)kTileCols, (cuuint64_t)kTileRows, n_kc, n_rg};
+    const cuuint64_t strides[3] = {(cuuint64_t)kTileCols * 2, (cuuint64_t)kTileBytes, n_kc * (cuuint64_t)kTileBytes};
+    const cuuint32_t box[4] = {(cuuint32_t)kTcBK, (cuuint32_t)kTileRows, 1, (cuuint32_t)(kTcBN / kTileRows)};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t*>(packed), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+               ? 0
+               : -1;
+}
+
+namespace {
+
+// ------------------------------------------------------------------------------------------ device: tcgen05 GEMM
+
+constexpr int kTcStages = 4;
+constexpr int kTcTile = kTcBM * kTcBK * 2;             // 16 KB: 128 rows x 128 bytes
+constexpr int kTcStageBytes = 3 * kTcTile;             // A_hi | A_lo | W
+constexpr int kTcThreads = 192;                        // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..5: epilogue
+constexpr int kTcTmemCols = kTcBN;                     // fp32 accumulator: 128 lanes x 128 columns
+constexpr int kTcSmem = kTcStages * kTcStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+enum : int { kErrTcFull = 11, kErrTcEmpty = 12, kErrTcAccum = 13 };
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile in the 128-byte-swizzle layout: rows of
+// 128 bytes, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t sw128_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128.
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(da), "l"(db), "r"(kTcIdesc), "r"(accumulate)
+        : "memory");
+}
+
+// arrives on the mbarrier once every matrix instruction issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive accumulator columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
+    hi = f32_to_bf16_bits(x);
+    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi));
+}
+
+// One CTA = one 128 x 128 tile of C.  CTAs with the same weight tile are neighbours in the grid, so
+// a weight tile comes from HBM once and from L2 for the other token tiles.
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant__ CUtensorMap tA_lo,
+               const __grid_constant__ CUtensorMap tW, const TcGemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
+    uint64_t* empty = full + kTcStages;
+    uint64_t* accum = empty + kTcStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_tiles = (g.m_rows + kTcBM - 1) / kTcBM;
+    const int m_tile = blockIdx.x % m_tiles, n_tile = blockIdx.x / m_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(accum, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) {   // the whole warp allocates the accumulator's TMEM columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < g.k_blocks; ++kb) {
+                const int s = kb % kTcStages;
+                if (kb >= kTcStages) mbar_wait(&empty[s], ((kb / kTcStages) - 1) & 1, g.err, kErrTcEmpty);
+                uint8_t* st = smem + s * kTcStageBytes;
+                mbar_arrive_expect_tx(&full[s], kTcStageBytes);
+                tma_load_2d(st, &tA_hi, kb * kTcBK, m_tile * kTcBM, &full[s]);
+                tma_load_2d(st + kTcTile, &tA_lo, kb * kTcBK, m_tile * kTcBM, &full[s]);
+                // packed weights: column chunk kb / 4, 64 columns at (kb % 4) * 64, row groups 4 n_tile ..
+                tma_load_4d(st + 2 * kTcTile, &tW, (kb % 4) * kTcBK, 0, kb / 4, n_tile * (kTcBN / kTileRows), &full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            for (int kb = 0; kb < g.k_blocks; ++kb) {
+                const int s = kb % kTcStages;
+                mbar_wait(&full[s], (kb / kTcStages) & 1, g.err, kErrTcFull);
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + s * kTcStageBytes);
+#pragma unroll
+                for (int k4 = 0; k4 < kTcBK / 16; ++k4) {
+                    // 16 columns = 32 bytes further along the swizzled 128-byte rows
+                    const uint64_t db = sw128_desc(sa + 2 * kTcTile + k4 * 32);
+                    umma_bf16(tmem_d, sw128_desc(sa + k4 * 32), db, (kb | k4) != 0);
+                    umma_bf16(tmem_d, sw128_desc(sa + kTcTile + k4 * 32), db, 1);
+                }
+                umma_commit(&empty[s]);     // the stage is free once these instructions have read it
+            }
+            umma_commit(accum);             // the accumulator is complete
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes 32 (w % 4) .. +31; lane = token row of the tile
+        const int quad = warp & 3;
+        mbar_wait(accum, 0, g.err, kErrTcAccum);
+        tc_fence_after();
+        const int row = m_tile * kTcBM + quad * 32 + lane;
+        const bool row_ok = row < g.m_rows;
+#pragma unroll 1
+        for (int cb = 0; cb < kTcBN / 32; ++cb) {
+            float v[32];
+            tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + cb * 32, v);
+            const int n0 = n_tile * kTcBN + cb * 32;
+            if (!row_ok) continue;
+            if (g.mode == kTcSwigluSplit) {
+                uint16_t* ph = g.out_hi + (size_t)row * g.ld_hl + (n0 >> 1);
+                uint16_t* pl = g.out_lo + (size_t)row * g.ld_hl + (n0 >> 1);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (n0 + 2 * j + 1 < g.n_cols) {
+                        const float gt = v[2 * j], up = v[2 * j + 1];
+                        uint16_t hi, lo;
+                        split_bf16((gt / (1.0f + expf(-gt))) * up, hi, lo);
+                        ph[j] = hi;
+                        pl[j] = lo;
+                    }
+                }
+            } else {
+                float* po = g.out + (size_t)row * g.ldo + n0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (n0 + j < g.n_cols) po[j] = (g.mode == kTcResid) ? po[j] + v[j] : v[j];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kTcTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------ small kernels
+
+__global__ void pf_embed_kernel(const uint16_t* __restrict__ E, const int* __restrict__ tokens, int D, float* __restrict__ h, int ldh) {
+    const int r = blockIdx.x;
+    const uint16_t* e = E + (size_t)tokens[r] * D;
+    for (int i = threadIdx.x; i < D; i += blockDim.x) h[(size_t)r * ldh + i] = bf16_bits_to_f32(e[i]);
+}
+
+__global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const float* __restrict__ gain, float eps, int D,
+                                     uint16_t* __restrict__ hi, uint16_t* __restrict__ lo, int ldx) {
+    __shared__ float red[32];
+    const int r = blockIdx.x;
+    const float* x = h + (size_t)r * ldh;
+    float inv = 1.f;
+    if (gain) {
+        float ssq = 0.f;
+        for (int i = threadIdx.x; i < D; i += blockDim.x) ssq = fmaf(x[i], x[i], ssq);
+        ssq = warp_sum(ssq);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ssq;
+        __syncthreads();
+        float tot = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+        inv = 1.0f / sqrtf(tot / (float)D + eps);
+    }
+    for (int i = threadIdx.x; i < D; i += blockDim.x) {
+        const float v = gain ? __fmul_rn(__fmul_rn(x[i], gain[i]), inv) : x[i];
+        uint16_t a, b;
+        split_bf16(v, a, b);
+        hi[(size_t)r * ldx + i] = a;
+        lo[(size_t)r * ldx + i] = b;
+    }
+}
+
+__global__ void pf_rope_kv_kernel(const PfKvArgs a) {
+    const int r = blockIdx.x;
+    const int pos = a.pos0 + r;
+    const int half = a.hd / 2;
+    float* q = a.qkv + (size_t)r * 3 * a.D;
+    const float* k = q + a.D;
+    const float* v = q + 2 * a.D;
+    const size_t page_elems = (size_t)2 * a.H * kPageTokens * a.hd;
+    uint16_t* pg = a.kv_layer + (size_t)a.page_table[pos / kPageTokens] * page_elems;
+    const float2* cs = a.rope + (size_t)pos * half;
+    for (int idx = threadIdx.x; idx < a.H * half; idx += blockDim.x) {
+        const int h = idx / half, i = idx - h * half;
+        const float2 c = cs[i];
+        const int d0 = h * a.hd + i, d1 = d0 + half;
+        const float q0 = q[d0], q1 = q[d1];
+        q[d0] = __fmaf_rn(q0, c.x, -__fmul_rn(q1, c.y));
+        q[d1] = __fmaf_rn(q1, c.x, __fmul_rn(q0, c.y));
+        const float k0 = k[d0], k1 = k[d1];
+        uint16_t* kd = pg + ((size_t)h * kPageTokens + (pos % kPageTokens)) * a.hd;
+        uint16_t* vd = kd + (size_t)a.H * kPageTokens * a.hd;
+        kd[i] = f32_to_bf16_bits(__fmaf_rn(k0, c.x, -__fmul_rn(k1, c.y)));
+        kd[i + half] = f32_to_bf16_bits(__fmaf_rn(k1, c.x, __fmul_rn(k0, c.y)));
+        vd[i] = f32_to_bf16_bits(v[d0]);
+        vd[i + half] = f32_to_bf16_bits(v[d1]);
+    }
+}
+
+// Causal attention for 64 query rows of one head per CTA: 4 threads per query, each owning a quarter
+// of the head dimension; K/V pages of 64 positions pass through shared memory; scores in blocks of
+// 16 keys with an online softmax in log2 units.
+template <int HD>
+__global__ void __launch_bounds__(256) pf_attn_kernel(const PfAttnArgs a) {
+    constexpr int QD = HD / 4;                 // dims per thread
+    __shared__ __align__(16) uint16_t ks[kPageTokens * HD];
+    __shared__ __align__(16) uint16_t vs[kPageTokens * HD];
+    const int h = blockIdx.y;
+    const int ql = threadIdx.x >> 2, part = threadIdx.x & 3;
+    const int r = blockIdx.x * 64 + ql;
+    const bool r_ok = r < a.rows;
+    const int pos = a.pos0 + r;
+    const float sscale = 1.4426950408889634f / sqrtf((float)HD);
+    float q[QD], o[QD];
+#pragma unroll
+    for (int j = 0; j < QD; ++j) {
+        q[j] = r_ok ? a.qkv[(size_t)r * 3 * a.D + h * HD + part * QD + j] * sscale : 0.f;
+        o[j] = 0.f;
+    }
+    float mx = __int_as_float(0xFF800000), den = 0.f;
+    const int last_row = min(a.rows, blockIdx.x * 64 + 64) - 1;
+    const int last_pos = a.pos0 + last_row;
+    const size_t page_elems = (size_t)2 * a.H * kPageTokens * HD;
+    for (int s = 0; s * kPageTokens <= last_pos; ++s) {
+        const uint16_t* pg = a.kv_layer + (size_t)a.page_table[s] * page_elems + (size_t)h * kPageTokens * HD;
+        const uint4* gk = reinterpret_cast<const uint4*>(pg);
+        const uint4* gv = reinterpret_cast<const uint4*>(pg + (size_t)a.H * kPageTokens * HD);
+        __syncthreads();
+        for (int i = threadIdx.x; i < kPageTokens * HD / 8; i += 256) {
+            reinterpret_cast<uint4*>(ks)[i] = gk[i];
+            reinterpret_cast<uint4*>(vs)[i] = gv[i];
+        }
+        __syncthreads();
+#pragma unroll 1
+        for (int b16 = 0; b16 < kPageTokens / 16; ++b16) {
+            const int kp0 = s * kPageTokens + b16 * 16;
+            if (!__any_sync(0xFFFFFFFFu, r_ok && kp0 <= pos)) continue;
+            float sc[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint4* kr = reinterpret_cast<const uint4*>(ks + (b16 * 16 + i) * HD + part * QD);
+                float d = 0.f;
+#pragma unroll
+                for (int j8 = 0; j8 < QD / 8; ++j8) {
+                    const uint4 kk = kr[j8];
+                    d = fmaf(q[j8 * 8 + 0], bf16_lo(kk.x), d); d = fmaf(q[j8 * 8 + 1], bf16_hi(kk.x), d);
+                    d = fmaf(q[j8 * 8 + 2], bf16_lo(kk.y), d); d = fmaf(q[j8 * 8 + 3], bf16_hi(kk.y), d);
+                    d = fmaf(q[j8 * 8 + 4], bf16_lo(kk.z), d); d = fmaf(q[j8 * 8 + 5], bf16_hi(kk.z), d);
+                    d = fmaf(q[j8 * 8 + 6], bf16_lo(kk.w), d); d = fmaf(q[j8 * 8 + 7], bf16_hi(kk.w), d);
+                }
+                d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
+                d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
+                sc[i] = (r_ok && kp0 + i <= pos) ? d : __int_as_float(0xFF800000);
+            }
+            float bm = sc[0];
+#pragma unroll
+            for (int i = 1; i < 16; ++i) bm = fmaxf(bm, sc[i]);
+            if (bm == __int_as_float(0xFF800000)) continue;     // nothing visible to this query in the block
+            const float nm = fmaxf(mx, bm);
+            const float corr = exp2f(mx - nm);
+            den *= corr;
+#pragma unroll
+            for (int j = 0; j < QD; ++j) o[j] *= corr;
+            mx = nm;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if (sc[i] == __int_as_float(0xFF800000)) continue;
+                const float p = exp2f(sc[i] - nm);
+                den += p;
+                const uint4* vr = reinterpret_cast<const uint4*>(vs + (b16 * 16 + i) * HD + part * QD);
+#pragma unroll
+                for (int j8 = 0; j8 < QD / 8; ++j8) {
+                    const uint4 vv = vr[j8];
+                    o[j8 * 8 + 0] = fmaf(p, bf16_lo(vv.x), o[j8 * 8 + 0]); o[j8 * 8 + 1] = fmaf(p, bf16_hi(vv.x), o[j8 * 8 + 1]);
+                    o[j8 * 8 + 2] = fmaf(p, bf16_lo(vv.y), o[j8 * 8 + 2]); o[j8 * 8 + 3] = fmaf(p, bf16_hi(vv.y), o[j8 * 8 + 3]);
+                    o[j8 * 8 + 4] = fmaf(p, bf16_lo(vv.z), o[j8 * 8 + 4]); o[j8 * 8 + 5] = fmaf(p, bf16_hi(vv.z), o[j8 * 8 + 5]);
+                    o[j8 * 8 + 6] = fmaf(p, bf16_lo(vv.w), o[j8 * 8 + 6]); o[j8 * 8 + 7] = fmaf(p, bf16_hi(vv.w), o[j8 * 8 + 7]);
+                }
+            }
+        }
+    }
+    if (r_ok) {
+        const float inv = 1.0f / den;
+#pragma unroll
+        for (int j = 0; j < QD; ++j) {
+            uint16_t hi, lo;
+            split_bf16(o[j] * inv, hi, lo);
+            const size_t at = (size_t)r * a.ld + h * HD + part * QD + j;
+            a.out_hi[at] = hi;
+            a.out_lo[at] = lo;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_lo, const CUtensorMap& w, const TcGemmArgs& g,
+                           cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (g.m_rows < 1 || g.n_cols < 1 || g.k_blocks < 1) return cudaErrorInvalidValue;
+    const int m_tiles = (g.m_rows + kTcBM - 1) / kTcBM, n_tiles = (g.n_cols + kTcBN - 1) / kTcBN;
+    tc_gemm_kernel<<<m_tiles * n_tiles, kTcThreads, kTcSmem, st>>>(a_hi, a_lo, w, g);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int D, float* h, int ldh, cudaStream_t st) {
+    pf_embed_kernel<<<rows, 256, 0, st>>>(E, tokens, D, h, ldh);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
+                                 uint16_t* lo, int ldx, cudaStream_t st) {
+    pf_norm_split_kernel<<<rows, 256, 0, st>>>(h, ldh, gain, eps, D, hi, lo, ldx);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pf_rope_kv(const PfKvArgs& a, cudaStream_t st) {
+    pf_rope_kv_kernel<<<a.rows, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pf_attn(const PfAttnArgs& a, cudaStream_t st) {
+    const dim3 grid((a.rows + 63) / 64, a.H);
+    if (a.hd == 128) pf_attn_kernel<128><<<grid, 256, 0, st>>>(a);
+    else if (a.hd == 64) pf_attn_kernel<64><<<grid, 256, 0, st>>>(a);
+    else return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+}  // namespace ppd

@@ -1,0 +1,74 @@
+// Prompt processing on the tensor cores (internal header).
+//
+// The prompt tokens before the start token ("forwarding with x<=t" ahead of the first step of
+// Algorithm 1) are independent rows of the same matrix products the decode step runs one row at a
+// time -- the only dense contraction of the method.  Here they go through tcgen05 matrix
+// instructions with the accumulator in tensor memory, fed by TMA tensor copies.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ppd {
+
+constexpr int kTcBM = 128;   // token rows per tile
+constexpr int kTcBN = 128;   // weight rows per tile (four packed row groups)
+constexpr int kTcBK = 64;    // columns per pipeline stage (128 bytes of bf16: one swizzle row)
+
+enum TcMode : int { kTcStore = 0, kTcResid = 1, kTcSwigluSplit = 2 };
+
+struct TcGemmArgs {
+    int m_rows;              // valid token rows
+    int n_cols;              // valid output columns (weight rows N)
+    int k_blocks;            // ceil(K / 64)
+    int mode;                // TcMode
+    float* out;              // kTcStore: C[m][n];  kTcResid: out[m][n] += C[m][n]
+    long long ldo;
+    uint16_t *out_hi, *out_lo;   // kTcSwigluSplit: silu(C[m][2j]) * C[m][2j+1] as bf16 hi + lo at [m][j]
+    long long ld_hl;
+    int* err;                // device error word (bounded waits)
+};
+
+// Resolves the driver's tensor-map encoder through the runtime (no link against the driver library).
+int tc_init();
+// 2-D map over row-major bf16 [rows][cols] (cols a multiple of 64), box 64 x 128, 128-byte swizzle.
+int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols);
+// 4-D map over a packed weight matrix ([row group][column chunk][32][256]), box = 64 columns of
+// four consecutive row groups: 128 weight rows x 128 bytes, 128-byte swizzle.
+int tc_map_packed(CUtensorMap* map, const uint16_t* packed, int n_rows, int n_cols);
+
+// C[m][n] = sum_k (A_hi + A_lo)[m][k] * W[n][k], fp32 accumulation in tensor memory.
+cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_lo, const CUtensorMap& w, const TcGemmArgs& g,
+                           cudaStream_t st);
+
+// h[r][:] = E[tokens[r]][:]
+cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int D, float* h, int ldh, cudaStream_t st);
+// x = gain ? RMSNorm(h; gain, eps) : h, written as bf16 hi + lo (x ~= hi + lo to about 2^-17 relative)
+cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
+                                 uint16_t* lo, int ldx, cudaStream_t st);
+
+struct PfKvArgs {
+    float* qkv;              // [rows][3D]: q is rotated in place; k, v are read
+    int rows, H, hd, D;
+    int pos0;                // position of row 0
+    const float2* rope;
+    uint16_t* kv_layer;      // this layer's pages
+    const int* page_table;
+};
+// rotary embedding of q and k at positions pos0 + r; k and v rounded to bf16 into the paged cache
+cudaError_t launch_pf_rope_kv(const PfKvArgs& a, cudaStream_t st);
+
+struct PfAttnArgs {
+    const float* qkv;        // rotated q at [r][h*hd ..]
+    int rows, H, hd, D;
+    int pos0;
+    const uint16_t* kv_layer;
+    const int* page_table;
+    uint16_t *out_hi, *out_lo;   // attention output as bf16 hi + lo, [rows][ld]
+    int ld;
+};
+// causal attention of rows at positions pos0 + r over cache positions 0 .. pos0 + r
+cudaError_t launch_pf_attn(const PfAttnArgs& a, cudaStream_t st);
+
+}  // namespace ppd

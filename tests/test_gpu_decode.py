@@ -379,3 +379,42 @@ def test_7b_full_depth_sampled_steps_against_oracle():
         assert ph[s] == int(p[s] in oracle_topk(pel[s], 3))
     ctx.close()
     print("7B sampled parity:", r, "hits", int(ph.sum()), "/ 24")
+
+
+@pytest.mark.parametrize("n_prompt", [2, 17, 130, 300])
+def test_tensor_core_prefill_against_oracle(tiny_shape, tiny_blob, n_prompt):
+    """The prompt through the tcgen05 matrix products and the causal attention kernel: decode
+    logits after it against the oracle (which prefills token by token in double precision), and
+    against the step-kernel prefill; PPD stays equal to greedy.  Lengths cover less than one tile
+    row block, a ragged second block and several KV pages."""
+    prompt = ppd_inputs.gen_prompt(tiny_shape.vocab, n_prompt, seed=31)
+    ctx = ppd.Context(tiny_shape, max_seq=360, max_k=3)
+    ctx.load_weights(tiny_blob)
+    ctx.set_prefill_chunk(4)
+    ctx.prefill(prompt)
+    ctx.step(3, 2)
+    ref = ctx.debug_logits()
+    ctx.set_prefill_chunk(0)
+    ctx.prefill(prompt)
+    ctx.step(3, 2)
+    assert np.abs(ctx.debug_logits() - ref).max() < 1e-4
+    check_against_oracle(tiny_shape, tiny_blob, prompt, 10, 3, 2, ctx=ctx, max_k=3)
+    ctx.prefill(prompt)
+    g, _ = ctx.decode(0, 0, 20)
+    ctx.prefill(prompt)
+    p, _ = ctx.decode(3, 2, 20)
+    assert (p == g).all()
+    ctx.close()
+
+
+def test_tensor_core_prefill_7b_shapes_two_layers():
+    """Full-width shapes (head dim 128, F = 11008: a K that ends inside a 256-column weight tile)
+    on a prompt longer than one 128-row tile."""
+    shape = ppd_inputs.LLAMA_7B.with_layers(2)
+    blob = ppd_inputs.gen_weights(shape, seed=0)
+    prompt = ppd_inputs.gen_prompt(shape.vocab, 150, seed=3)
+    ctx = ppd.Context(shape, max_seq=256, max_k=3)
+    ctx.load_weights(blob)
+    ctx.set_prefill_chunk(0)
+    check_against_oracle(shape, blob, prompt, 3, 3, 1, ctx=ctx, max_k=3)
+    ctx.close()

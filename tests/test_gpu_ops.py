@@ -217,3 +217,24 @@ def test_attention_rows_do_not_depend_on_M_and_long_prefix():
     # canonical tail (cache) and slot tail give the same bits
     c = _attention_case(2, 128, 8191, 1, seed=3, use_slots=False, permute=True)
     assert (c[0] == b[0]).all()
+
+
+@pytest.mark.parametrize("N,K,M", [(768, 256, 5), (1376, 256, 130), (256, 688, 200), (4096, 1024, 300)])
+def test_tensor_core_gemm_against_oracle(N, K, M):
+    """The prompt path's many-row product (tcgen05, bf16 hi + lo activations) against the oracle's
+    double-precision matvec, row by row on sampled rows; tiles, ragged rows and a K that is not a
+    multiple of the 64-column pipeline block are covered."""
+    rng = np.random.default_rng(N + 7 * K + 13 * M)
+    w = bf16_bits(rng, (N, K), 0.05)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    wp = pack(w)
+    xd = torch.from_numpy(x).to(DEV)
+    out = torch.full((M, N + 5), 7.0, dtype=torch.float32, device=DEV)
+    scratch = torch.empty(ppd.op_gemm_scratch_bytes(M, K), dtype=torch.uint8, device=DEV)
+    ppd.op_gemm(wp, N, K, xd, out, scratch)
+    got = out.cpu().numpy()
+    assert (got[:, N:] == 7.0).all()
+    for m in sorted(set([0, 1, M // 2, M - 1, min(M - 1, 127), min(M - 1, 128)])):
+        ref = oracle.matvec(w, x[m].astype(np.float64))
+        scale = np.abs(ref).max() + 1e-6
+        assert np.abs(got[m, :N] - ref).max() < 3e-5 * scale + 1e-6, m
