@@ -105,15 +105,16 @@ int ppd_set_sampling(ppd_ctx* ctx, int32_t top_k, float temperature, const float
 
 /* Fills the KV cache from a prompt (host, n_prompt >= 1 ids in [0, vocab)).  The last prompt
  * token is the start token x_0 of Algorithm 1: positions 0..n_prompt-2 are cached and
- * prompt[n_prompt-1] stays pending for the first decode step.  Resets the position.  In the default
- * mode the prompt runs through the step kernel in chunks of 4 tokens per launch. */
+ * prompt[n_prompt-1] stays pending for the first decode step.  Resets the position.  By default the
+ * prompt rows run on the tensor cores (see ppd_set_prefill_chunk). */
 int ppd_prefill(ppd_ctx* ctx, const int32_t* prompt, int32_t n_prompt);
 
 /* How ppd_prefill processes the prompt.
- *   n_tokens = 4 (default), 8, 2 or 1: through the step kernel, that many prompt tokens per launch;
- *     the tokens of a chunk share one pass over the weights and attend causally to each other.
- *   n_tokens = 0: on the tensor cores -- the prompt rows (up to 1024 per pass) go through tcgen05
- *     matrix products (activations as bf16 hi + lo pairs, fp32 accumulation) and a causal
+ *   n_tokens = 4, 8, 2 or 1: through the step kernel, that many prompt tokens per launch; the
+ *     tokens of a chunk share one pass over the weights and attend causally to each other.
+ *   n_tokens = 0 (default): on the tensor cores -- the prompt rows (up to 1024 per pass) go through tcgen05
+ *     matrix products (each float activation as three bf16 terms that sum to it exactly, fp32
+ *     accumulation) and a causal
  *     attention kernel over the paged cache.  The paper only says that the prompt is forwarded
  *     ("x<=t" in Algorithm 1); this is the one dense contraction of the method.
  * All settings differ in float rounding only. */
@@ -210,8 +211,8 @@ int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int3
                 int32_t ldo, void* stream);
 
 /* Many-row matrix product on the tensor cores (the prompt path's building block):
- * out[m][n] = sum_k W[n][k] x[m][k] for m < M (any M >= 1), fp32 accumulation, x split into bf16
- * hi + lo pairs.  w_packed: device, packed [N][K].  x: device float32 [M][ldx].  out: device
+ * out[m][n] = sum_k W[n][k] x[m][k] for m < M (any M >= 1), fp32 accumulation, x split into three
+ * bf16 terms that sum to it exactly.  w_packed: device, packed [N][K].  x: device float32 [M][ldx].  out: device
  * float32 [M][ldo].  scratch: device, >= ppd_op_gemm_scratch_bytes(M, K) bytes, 256-byte aligned.
  * Synchronises the stream; PPD_ETIMEOUT if a bounded device wait gave up. */
 size_t ppd_op_gemm_scratch_bytes(int32_t M, int32_t K);

@@ -38,7 +38,7 @@ struct Layout {
     size_t ws_h, ws_qkv, ws_attn, ws_z, ws_part, ws_tick, ws_bytes[2];   // offsets inside a workspace
     size_t logits_final, logits_early, top_final, top_early, head_scratch;
     size_t state, sample_u, prompt, out_tokens, out_hit, out_margin, timeline, staging, total;
-    size_t pf_h, pf_qkv, pf_xhi, pf_xlo, pf_zhi, pf_zlo;   // tensor-core prompt path: activations of up to pf_rows tokens
+    size_t pf_h, pf_qkv, pf_xhi, pf_xmid, pf_xlo, pf_zhi, pf_zmid, pf_zlo;   // tensor-core prompt path: activations of up to pf_rows tokens
     int pf_rows;
 };
 
@@ -121,8 +121,10 @@ Layout plan(const ppd_config& c) {
         L.pf_h = take((size_t)L.pf_rows * L.Dp * 4);
         L.pf_qkv = take((size_t)L.pf_rows * 3 * D * 4);
         L.pf_xhi = take((size_t)L.pf_rows * L.Dp * 2);
+        L.pf_xmid = take((size_t)L.pf_rows * L.Dp * 2);
         L.pf_xlo = take((size_t)L.pf_rows * L.Dp * 2);
         L.pf_zhi = take((size_t)L.pf_rows * L.Fp * 2);
+        L.pf_zmid = take((size_t)L.pf_rows * L.Fp * 2);
         L.pf_zlo = take((size_t)L.pf_rows * L.Fp * 2);
     }
     L.total = o;
@@ -155,7 +157,7 @@ struct ppd_ctx {
     bool trace;                       // record per-phase timestamps of the fused kernel
     int prefill_chunk;                // prompt tokens per prefill launch (1, 2, 4 or 8); 0 = tensor-core path
     bool tc_ok;                       // tensor maps of the tensor-core prompt path are ready
-    CUtensorMap map_xhi, map_xlo, map_zhi, map_zlo;
+    CUtensorMap map_xhi, map_xmid, map_xlo, map_zhi, map_zmid, map_zlo;
     std::vector<CUtensorMap> map_w;   // per layer: Wqkv, Wo, Wgu, Wd
     int sample_k, n_sample_u;         // top-k sampling of the final prediction (0 = greedy)
     float temperature;
@@ -492,8 +494,8 @@ int prefill_tc(ppd_ctx* x, int n_prompt) {
     const int D = c.d_model, F = c.d_ffn;
     float* h = at<float>(x, L.pf_h);
     float* qkv = at<float>(x, L.pf_qkv);
-    uint16_t *xhi = at<uint16_t>(x, L.pf_xhi), *xlo = at<uint16_t>(x, L.pf_xlo);
-    uint16_t *zhi = at<uint16_t>(x, L.pf_zhi), *zlo = at<uint16_t>(x, L.pf_zlo);
+    uint16_t *xhi = at<uint16_t>(x, L.pf_xhi), *xmid = at<uint16_t>(x, L.pf_xmid), *xlo = at<uint16_t>(x, L.pf_xlo);
+    uint16_t *zhi = at<uint16_t>(x, L.pf_zhi), *zmid = at<uint16_t>(x, L.pf_zmid), *zlo = at<uint16_t>(x, L.pf_zlo);
     for (int t0 = 0; t0 + 1 < n_prompt; t0 += L.pf_rows) {
         const int m = n_prompt - 1 - t0 < L.pf_rows ? n_prompt - 1 - t0 : L.pf_rows;
         CK(launch_pf_embed(at<uint16_t>(x, L.emb), at<int>(x, L.prompt) + t0, m, D, h, L.Dp, x->sm));
@@ -503,9 +505,9 @@ int prefill_tc(ppd_ctx* x, int n_prompt) {
             TcGemmArgs g{};
             g.m_rows = m;
             g.err = x->state + S_ERR;
-            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g1), c.rms_eps, m, D, xhi, xlo, L.Dp, x->sm));
+            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g1), c.rms_eps, m, D, xhi, xmid, xlo, L.Dp, x->sm));
             g.n_cols = 3 * D; g.k_blocks = (D + kTcBK - 1) / kTcBK; g.mode = kTcStore; g.out = qkv; g.ldo = 3 * D;
-            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[0], g, x->sm));
+            CK(launch_tc_gemm(x->map_xhi, x->map_xmid, x->map_xlo, mw[0], g, x->sm));
             PfKvArgs kv{};
             kv.qkv = qkv; kv.rows = m; kv.H = c.n_heads; kv.hd = c.head_dim; kv.D = D; kv.pos0 = t0;
             kv.rope = at<float2>(x, L.rope);
@@ -514,15 +516,15 @@ int prefill_tc(ppd_ctx* x, int n_prompt) {
             CK(launch_pf_rope_kv(kv, x->sm));
             PfAttnArgs pa{};
             pa.qkv = qkv; pa.rows = m; pa.H = c.n_heads; pa.hd = c.head_dim; pa.D = D; pa.pos0 = t0;
-            pa.kv_layer = kv.kv_layer; pa.page_table = kv.page_table; pa.out_hi = xhi; pa.out_lo = xlo; pa.ld = L.Dp;
+            pa.kv_layer = kv.kv_layer; pa.page_table = kv.page_table; pa.out_hi = xhi; pa.out_mid = xmid; pa.out_lo = xlo; pa.ld = L.Dp;
             CK(launch_pf_attn(pa, x->sm));
             g.n_cols = D; g.mode = kTcResid; g.out = h; g.ldo = L.Dp;
-            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[1], g, x->sm));
-            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g2), c.rms_eps, m, D, xhi, xlo, L.Dp, x->sm));
-            g.n_cols = 2 * F; g.mode = kTcSwigluSplit; g.out = nullptr; g.out_hi = zhi; g.out_lo = zlo; g.ld_hl = L.Fp;
-            CK(launch_tc_gemm(x->map_xhi, x->map_xlo, mw[2], g, x->sm));
+            CK(launch_tc_gemm(x->map_xhi, x->map_xmid, x->map_xlo, mw[1], g, x->sm));
+            CK(launch_pf_norm_split(h, L.Dp, reinterpret_cast<const float*>(lb + L.off_g2), c.rms_eps, m, D, xhi, xmid, xlo, L.Dp, x->sm));
+            g.n_cols = 2 * F; g.mode = kTcSwigluSplit; g.out = nullptr; g.out_hi = zhi; g.out_mid = zmid; g.out_lo = zlo; g.ld_hl = L.Fp;
+            CK(launch_tc_gemm(x->map_xhi, x->map_xmid, x->map_xlo, mw[2], g, x->sm));
             g.n_cols = D; g.k_blocks = (F + kTcBK - 1) / kTcBK; g.mode = kTcResid; g.out = h; g.ldo = L.Dp;
-            CK(launch_tc_gemm(x->map_zhi, x->map_zlo, mw[3], g, x->sm));
+            CK(launch_tc_gemm(x->map_zhi, x->map_zmid, x->map_zlo, mw[3], g, x->sm));
         }
     }
     return PPD_OK;
@@ -573,7 +575,7 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     x->pdl = true;
     x->fused = true;
     x->w_early = nullptr;
-    x->prefill_chunk = 4;
+    x->prefill_chunk = 4;      // replaced by 0 (tensor-core path) below once its tensor maps exist
     x->sample_k = 0; x->n_sample_u = 0; x->temperature = 1.f;
     x->trace = false;
     x->pos = 0; x->pending = -1; x->prev_hit = false; x->prev_b = 0;
@@ -616,8 +618,10 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
     if (x->tc_ok) {
         const int D = cfg->d_model, F = cfg->d_ffn;
         x->tc_ok = tc_map_rows(&x->map_xhi, at<uint16_t>(x, L.pf_xhi), L.pf_rows, L.Dp) == 0 &&
+                   tc_map_rows(&x->map_xmid, at<uint16_t>(x, L.pf_xmid), L.pf_rows, L.Dp) == 0 &&
                    tc_map_rows(&x->map_xlo, at<uint16_t>(x, L.pf_xlo), L.pf_rows, L.Dp) == 0 &&
                    tc_map_rows(&x->map_zhi, at<uint16_t>(x, L.pf_zhi), L.pf_rows, L.Fp) == 0 &&
+                   tc_map_rows(&x->map_zmid, at<uint16_t>(x, L.pf_zmid), L.pf_rows, L.Fp) == 0 &&
                    tc_map_rows(&x->map_zlo, at<uint16_t>(x, L.pf_zlo), L.pf_rows, L.Fp) == 0;
         x->map_w.resize((size_t)cfg->n_layers * 4);
         for (int l = 0; l < cfg->n_layers && x->tc_ok; ++l) {
@@ -629,6 +633,7 @@ int ppd_create(const ppd_config* cfg, void* dev_mem, size_t dev_bytes, void* str
                        tc_map_packed(&mw[3], reinterpret_cast<uint16_t*>(lb + L.off_wd), D, F) == 0;
         }
     }
+    if (x->tc_ok) x->prefill_chunk = 0;
     *out = x;
     return PPD_OK;
 }
@@ -995,7 +1000,7 @@ int ppd_op_gemv(const void* w_packed, int32_t N, int32_t K, const float* x, int3
 
 size_t ppd_op_gemm_scratch_bytes(int32_t M, int32_t K) {
     if (M < 1 || K < 1) return 0;
-    return (size_t)2 * round_up(M, kTcBM) * round_up(K, kTileCols) * 2 + 256;
+    return (size_t)3 * round_up(M, kTcBM) * round_up(K, kTileCols) * 2 + 256;
 }
 
 int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, float* out,
@@ -1008,16 +1013,17 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
     const int Mp = (int)round_up(M, kTcBM), Kp = (int)round_up(K, kTileCols);
     int* err = reinterpret_cast<int*>(scratch);
     uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256);
-    uint16_t* lo = hi + (size_t)Mp * Kp;
+    uint16_t* mid = hi + (size_t)Mp * Kp;
+    uint16_t* lo = mid + (size_t)Mp * Kp;
     CKOP(cudaMemsetAsync(scratch, 0, ppd_op_gemm_scratch_bytes(M, K), st));
-    CKOP(launch_pf_norm_split(x, ldx, nullptr, 0.f, M, K, hi, lo, Kp, st));
-    CUtensorMap ma, mb, mw;
-    if (tc_map_rows(&ma, hi, Mp, Kp) || tc_map_rows(&mb, lo, Mp, Kp) ||
+    CKOP(launch_pf_norm_split(x, ldx, nullptr, 0.f, M, K, hi, mid, lo, Kp, st));
+    CUtensorMap ma, mm, mb, mw;
+    if (tc_map_rows(&ma, hi, Mp, Kp) || tc_map_rows(&mm, mid, Mp, Kp) || tc_map_rows(&mb, lo, Mp, Kp) ||
         tc_map_packed(&mw, reinterpret_cast<const uint16_t*>(w_packed), N, K))
         return PPD_ECUDA;
     TcGemmArgs g{};
     g.m_rows = M; g.n_cols = N; g.k_blocks = (K + kTcBK - 1) / kTcBK; g.mode = kTcStore; g.out = out; g.ldo = ldo; g.err = err;
-    CKOP(launch_tc_gemm(ma, mb, mw, g, st));
+    CKOP(launch_tc_gemm(ma, mm, mb, mw, g, st));
     int h_err = 0;
     CKOP(cudaMemcpyAsync(&h_err, err, 4, cudaMemcpyDeviceToHost, st));
     CKOP(cudaStreamSynchronize(st));

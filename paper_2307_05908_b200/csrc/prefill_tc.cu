@@ -1,11 +1,13 @@
 // Prompt processing on the tensor cores: tcgen05 matrix products with the accumulator in tensor
 // memory, operands staged by TMA tensor copies, plus the small kernels around them (embedding rows,
-// RMSNorm + bf16 hi/lo split, rotary embedding + KV write, causal attention over the paged cache).
+// RMSNorm + bf16 hi/mid/lo split, rotary embedding + KV write, causal attention over the paged cache).
 //
 // Precision: the weights are bf16 already; an activation x (fp32) enters the tensor cores as the
-// pair hi = bf16(x), lo = bf16(x - hi), two matrix instructions per tile, so x is represented to
-// about 2^-17 relative and the products are exact in the fp32 accumulator.  This keeps the prompt's
-// K/V and hidden states within float rounding of the decode path's.
+// triple hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid) -- three 8-bit mantissas hold the
+// 24 bits of a float exactly -- with three matrix instructions per tile, so every product is exact
+// and only the fp32 accumulation rounds.  A two-way split (2^-18 relative per activation) was not
+// enough: it moved about 0.2 % of the prompt's K/V elements across a bf16 rounding boundary, which
+// after 32 layers showed up as logit differences above the 2e-2 parity bound.
 #include "common.cuh"
 #include "prefill_tc.cuh"
 
@@ -62,11 +64,11 @@ namespace {
 
 // ------------------------------------------------------------------------------------------ device: tcgen05 GEMM
 
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 3;
 constexpr int kTcTile = kTcBM * kTcBK * 2;             // 16 KB: 128 rows x 128 bytes
-constexpr int kTcStageBytes = 3 * kTcTile;             // A_hi | A_lo | W
+constexpr int kTcStageBytes = 4 * kTcTile;             // A_hi | A_mid | A_lo | W
 constexpr int kTcThreads = 192;                        // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..5: epilogue
-constexpr int kTcTmemCols = kTcBN;                     // fp32 accumulator: 128 lanes x 128 columns
+constexpr int kTcTmemCols = 2 * kTcBN;                 // two fp32 accumulator buffers: 128 lanes x 128 columns each
 constexpr int kTcSmem = kTcStages * kTcStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 enum : int { kErrTcFull = 11, kErrTcEmpty = 12, kErrTcAccum = 13 };
 
@@ -130,22 +132,31 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
+__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& mid, uint16_t& lo) {
     hi = f32_to_bf16_bits(x);
-    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi));
+    const float r1 = x - bf16_bits_to_f32(hi);       // exact
+    mid = f32_to_bf16_bits(r1);
+    lo = f32_to_bf16_bits(r1 - bf16_bits_to_f32(mid));   // exact, and the remainder fits 8 bits
 }
 
 // One CTA = one 128 x 128 tile of C.  CTAs with the same weight tile are neighbours in the grid, so
 // a weight tile comes from HBM once and from L2 for the other token tiles.
+//
+// The tensor core adds into its fp32 accumulator with truncation, not round-to-nearest: over the
+// hundreds of matrix instructions of a long K the error grows linearly (measured: 1.4e-5 relative
+// at K = 4096), far above a float dot product's.  So the accumulator in tensor memory only ever holds
+// ONE 64-column block of K (12 instructions); the epilogue warps drain it into fp32 registers with
+// ordinary rounded adds while the next block accumulates into the other of two TMEM buffers.
 __global__ void __launch_bounds__(kTcThreads, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant__ CUtensorMap tA_lo,
-               const __grid_constant__ CUtensorMap tW, const TcGemmArgs g) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant__ CUtensorMap tA_mid,
+               const __grid_constant__ CUtensorMap tA_lo, const __grid_constant__ CUtensorMap tW, const TcGemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
     uint64_t* empty = full + kTcStages;
-    uint64_t* accum = empty + kTcStages;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+    uint64_t* tfull = empty + kTcStages;     // [2] a TMEM buffer holds a finished block
+    uint64_t* tempty = tfull + 2;            // [2] the epilogue warps have drained it
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m_tiles = (g.m_rows + kTcBM - 1) / kTcBM;
@@ -156,10 +167,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(accum, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&tfull[b], 1);
+            mbar_init(&tempty[b], 4);        // one arrival per epilogue warp
+        }
         fence_barrier_init();
     }
-    if (warp == 1) {   // the whole warp allocates the accumulator's TMEM columns
+    if (warp == 1) {   // the whole warp allocates the two accumulator buffers
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTcTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -177,60 +191,77 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
                 uint8_t* st = smem + s * kTcStageBytes;
                 mbar_arrive_expect_tx(&full[s], kTcStageBytes);
                 tma_load_2d(st, &tA_hi, kb * kTcBK, m_tile * kTcBM, &full[s]);
-                tma_load_2d(st + kTcTile, &tA_lo, kb * kTcBK, m_tile * kTcBM, &full[s]);
+                tma_load_2d(st + kTcTile, &tA_mid, kb * kTcBK, m_tile * kTcBM, &full[s]);
+                tma_load_2d(st + 2 * kTcTile, &tA_lo, kb * kTcBK, m_tile * kTcBM, &full[s]);
                 // packed weights: column chunk kb / 4, 64 columns at (kb % 4) * 64, row groups 4 n_tile ..
-                tma_load_4d(st + 2 * kTcTile, &tW, (kb % 4) * kTcBK, 0, kb / 4, n_tile * (kTcBN / kTileRows), &full[s]);
+                tma_load_4d(st + 3 * kTcTile, &tW, (kb % 4) * kTcBK, 0, kb / 4, n_tile * (kTcBN / kTileRows), &full[s]);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             for (int kb = 0; kb < g.k_blocks; ++kb) {
-                const int s = kb % kTcStages;
+                const int s = kb % kTcStages, buf = kb & 1;
+                if (kb >= 2) mbar_wait(&tempty[buf], ((kb >> 1) - 1) & 1, g.err, kErrTcAccum);
                 mbar_wait(&full[s], (kb / kTcStages) & 1, g.err, kErrTcFull);
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + s * kTcStageBytes);
+                const uint32_t td = tmem_d + buf * kTcBN;
 #pragma unroll
                 for (int k4 = 0; k4 < kTcBK / 16; ++k4) {
                     // 16 columns = 32 bytes further along the swizzled 128-byte rows
-                    const uint64_t db = sw128_desc(sa + 2 * kTcTile + k4 * 32);
-                    umma_bf16(tmem_d, sw128_desc(sa + k4 * 32), db, (kb | k4) != 0);
-                    umma_bf16(tmem_d, sw128_desc(sa + kTcTile + k4 * 32), db, 1);
+                    const uint64_t db = sw128_desc(sa + 3 * kTcTile + k4 * 32);
+                    umma_bf16(td, sw128_desc(sa + k4 * 32), db, k4 != 0);
+                    umma_bf16(td, sw128_desc(sa + kTcTile + k4 * 32), db, 1);
+                    umma_bf16(td, sw128_desc(sa + 2 * kTcTile + k4 * 32), db, 1);
                 }
-                umma_commit(&empty[s]);     // the stage is free once these instructions have read it
+                umma_commit(&empty[s]);      // the stage is free once these instructions have read it
+                umma_commit(&tfull[buf]);    // and the block's sums are complete
             }
-            umma_commit(accum);             // the accumulator is complete
         }
     } else {
-        // epilogue: warp w may touch TMEM lanes 32 (w % 4) .. +31; lane = token row of the tile
+        // epilogue warps: warp w may touch TMEM lanes 32 (w % 4) .. +31; lane = token row of the tile
         const int quad = warp & 3;
-        mbar_wait(accum, 0, g.err, kErrTcAccum);
-        tc_fence_after();
+        float acc[kTcBN];
+#pragma unroll
+        for (int i = 0; i < kTcBN; ++i) acc[i] = 0.f;
+        for (int kb = 0; kb < g.k_blocks; ++kb) {
+            const int buf = kb & 1;
+            mbar_wait(&tfull[buf], (kb >> 1) & 1, g.err, kErrTcAccum);
+            tc_fence_after();
+#pragma unroll
+            for (int cb = 0; cb < kTcBN / 32; ++cb) {
+                float v[32];
+                tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kTcBN + cb * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) acc[cb * 32 + i] += v[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[buf]);
+        }
         const int row = m_tile * kTcBM + quad * 32 + lane;
-        const bool row_ok = row < g.m_rows;
-#pragma unroll 1
-        for (int cb = 0; cb < kTcBN / 32; ++cb) {
-            float v[32];
-            tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + cb * 32, v);
-            const int n0 = n_tile * kTcBN + cb * 32;
-            if (!row_ok) continue;
+        if (row < g.m_rows) {
+            const int n0 = n_tile * kTcBN;
             if (g.mode == kTcSwigluSplit) {
                 uint16_t* ph = g.out_hi + (size_t)row * g.ld_hl + (n0 >> 1);
+                uint16_t* pm = g.out_mid + (size_t)row * g.ld_hl + (n0 >> 1);
                 uint16_t* pl = g.out_lo + (size_t)row * g.ld_hl + (n0 >> 1);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
+                for (int j = 0; j < kTcBN / 2; ++j) {
                     if (n0 + 2 * j + 1 < g.n_cols) {
-                        const float gt = v[2 * j], up = v[2 * j + 1];
-                        uint16_t hi, lo;
-                        split_bf16((gt / (1.0f + expf(-gt))) * up, hi, lo);
+                        const float gt = acc[2 * j], up = acc[2 * j + 1];
+                        uint16_t hi, mid, lo;
+                        split_bf16((gt / (1.0f + expf(-gt))) * up, hi, mid, lo);
                         ph[j] = hi;
+                        pm[j] = mid;
                         pl[j] = lo;
                     }
                 }
             } else {
                 float* po = g.out + (size_t)row * g.ldo + n0;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if (n0 + j < g.n_cols) po[j] = (g.mode == kTcResid) ? po[j] + v[j] : v[j];
+                for (int j = 0; j < kTcBN; ++j) {
+                    if (n0 + j < g.n_cols) po[j] = (g.mode == kTcResid) ? po[j] + acc[j] : acc[j];
                 }
             }
         }
@@ -251,7 +282,7 @@ __global__ void pf_embed_kernel(const uint16_t* __restrict__ E, const int* __res
 }
 
 __global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const float* __restrict__ gain, float eps, int D,
-                                     uint16_t* __restrict__ hi, uint16_t* __restrict__ lo, int ldx) {
+                                     uint16_t* __restrict__ hi, uint16_t* __restrict__ mid, uint16_t* __restrict__ lo, int ldx) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const float* x = h + (size_t)r * ldh;
@@ -268,10 +299,11 @@ __global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const
     }
     for (int i = threadIdx.x; i < D; i += blockDim.x) {
         const float v = gain ? __fmul_rn(__fmul_rn(x[i], gain[i]), inv) : x[i];
-        uint16_t a, b;
-        split_bf16(v, a, b);
+        uint16_t a, b, c;
+        split_bf16(v, a, b, c);
         hi[(size_t)r * ldx + i] = a;
-        lo[(size_t)r * ldx + i] = b;
+        mid[(size_t)r * ldx + i] = b;
+        lo[(size_t)r * ldx + i] = c;
     }
 }
 
@@ -388,10 +420,11 @@ __global__ void __launch_bounds__(256) pf_attn_kernel(const PfAttnArgs a) {
         const float inv = 1.0f / den;
 #pragma unroll
         for (int j = 0; j < QD; ++j) {
-            uint16_t hi, lo;
-            split_bf16(o[j] * inv, hi, lo);
+            uint16_t hi, mid, lo;
+            split_bf16(o[j] * inv, hi, mid, lo);
             const size_t at = (size_t)r * a.ld + h * HD + part * QD + j;
             a.out_hi[at] = hi;
+            a.out_mid[at] = mid;
             a.out_lo[at] = lo;
         }
     }
@@ -399,8 +432,8 @@ __global__ void __launch_bounds__(256) pf_attn_kernel(const PfAttnArgs a) {
 
 }  // namespace
 
-cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_lo, const CUtensorMap& w, const TcGemmArgs& g,
-                           cudaStream_t st) {
+cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_mid, const CUtensorMap& a_lo, const CUtensorMap& w,
+                           const TcGemmArgs& g, cudaStream_t st) {
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
@@ -409,7 +442,7 @@ cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_lo, con
     }
     if (g.m_rows < 1 || g.n_cols < 1 || g.k_blocks < 1) return cudaErrorInvalidValue;
     const int m_tiles = (g.m_rows + kTcBM - 1) / kTcBM, n_tiles = (g.n_cols + kTcBN - 1) / kTcBN;
-    tc_gemm_kernel<<<m_tiles * n_tiles, kTcThreads, kTcSmem, st>>>(a_hi, a_lo, w, g);
+    tc_gemm_kernel<<<m_tiles * n_tiles, kTcThreads, kTcSmem, st>>>(a_hi, a_mid, a_lo, w, g);
     return cudaGetLastError();
 }
 
@@ -419,8 +452,8 @@ cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int 
 }
 
 cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
-                                 uint16_t* lo, int ldx, cudaStream_t st) {
-    pf_norm_split_kernel<<<rows, 256, 0, st>>>(h, ldh, gain, eps, D, hi, lo, ldx);
+                                 uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st) {
+    pf_norm_split_kernel<<<rows, 256, 0, st>>>(h, ldh, gain, eps, D, hi, mid, lo, ldx);
     return cudaGetLastError();
 }
 

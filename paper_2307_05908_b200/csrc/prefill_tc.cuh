@@ -25,7 +25,7 @@ struct TcGemmArgs {
     int mode;                // TcMode
     float* out;              // kTcStore: C[m][n];  kTcResid: out[m][n] += C[m][n]
     long long ldo;
-    uint16_t *out_hi, *out_lo;   // kTcSwigluSplit: silu(C[m][2j]) * C[m][2j+1] as bf16 hi + lo at [m][j]
+    uint16_t *out_hi, *out_mid, *out_lo;   // kTcSwigluSplit: silu(C[m][2j]) * C[m][2j+1] as bf16 hi + mid + lo at [m][j]
     long long ld_hl;
     int* err;                // device error word (bounded waits)
 };
@@ -38,15 +38,15 @@ int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols);
 // four consecutive row groups: 128 weight rows x 128 bytes, 128-byte swizzle.
 int tc_map_packed(CUtensorMap* map, const uint16_t* packed, int n_rows, int n_cols);
 
-// C[m][n] = sum_k (A_hi + A_lo)[m][k] * W[n][k], fp32 accumulation in tensor memory.
-cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_lo, const CUtensorMap& w, const TcGemmArgs& g,
-                           cudaStream_t st);
+// C[m][n] = sum_k (A_hi + A_mid + A_lo)[m][k] * W[n][k], fp32 accumulation in tensor memory.
+cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_mid, const CUtensorMap& a_lo, const CUtensorMap& w,
+                           const TcGemmArgs& g, cudaStream_t st);
 
 // h[r][:] = E[tokens[r]][:]
 cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int D, float* h, int ldh, cudaStream_t st);
-// x = gain ? RMSNorm(h; gain, eps) : h, written as bf16 hi + lo (x ~= hi + lo to about 2^-17 relative)
+// x = gain ? RMSNorm(h; gain, eps) : h, written as bf16 hi + mid + lo (their sum is x exactly)
 cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
-                                 uint16_t* lo, int ldx, cudaStream_t st);
+                                 uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st);
 
 struct PfKvArgs {
     float* qkv;              // [rows][3D]: q is rotated in place; k, v are read
@@ -65,7 +65,7 @@ struct PfAttnArgs {
     int pos0;
     const uint16_t* kv_layer;
     const int* page_table;
-    uint16_t *out_hi, *out_lo;   // attention output as bf16 hi + lo, [rows][ld]
+    uint16_t *out_hi, *out_mid, *out_lo;   // attention output as bf16 hi + mid + lo, [rows][ld]
     int ld;
 };
 // causal attention of rows at positions pos0 + r over cache positions 0 .. pos0 + r

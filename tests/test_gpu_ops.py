@@ -221,7 +221,7 @@ def test_attention_rows_do_not_depend_on_M_and_long_prefix():
 
 @pytest.mark.parametrize("N,K,M", [(768, 256, 5), (1376, 256, 130), (256, 688, 200), (4096, 1024, 300)])
 def test_tensor_core_gemm_against_oracle(N, K, M):
-    """The prompt path's many-row product (tcgen05, bf16 hi + lo activations) against the oracle's
+    """The prompt path's many-row product (tcgen05, each activation as three bf16 terms) against the oracle's
     double-precision matvec, row by row on sampled rows; tiles, ragged rows and a K that is not a
     multiple of the 64-column pipeline block are covered."""
     rng = np.random.default_rng(N + 7 * K + 13 * M)
