@@ -67,7 +67,8 @@ namespace {
 constexpr int kTcStages = 3;
 constexpr int kTcTile = kTcBM * kTcBK * 2;             // 16 KB: 128 rows x 128 bytes
 constexpr int kTcStageBytes = 4 * kTcTile;             // A_hi | A_mid | A_lo | W
-constexpr int kTcThreads = 192;                        // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..5: epilogue
+constexpr int kTcThreads = 320;                        // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..9: epilogue
+constexpr int kTcEpiCols = kTcBN / 2;                  // columns per epilogue warp: two warps share a TMEM lane quadrant
 constexpr int kTcTmemCols = 2 * kTcBN;                 // two fp32 accumulator buffers: 128 lanes x 128 columns each
 constexpr int kTcSmem = kTcStages * kTcStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 enum : int { kErrTcFull = 11, kErrTcEmpty = 12, kErrTcAccum = 13 };
@@ -114,9 +115,8 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 32 consecutive accumulator columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
+// 32 consecutive accumulator columns of this thread's TMEM lane; the caller waits (tcgen05.wait::ld)
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -127,9 +127,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& mid, uint16_t& lo) {
@@ -169,7 +166,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tfull[b], 1);
-            mbar_init(&tempty[b], 4);        // one arrival per epilogue warp
+            mbar_init(&tempty[b], 8);        // one arrival per epilogue warp
         }
         fence_barrier_init();
     }
@@ -219,21 +216,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
             }
         }
     } else {
-        // epilogue warps: warp w may touch TMEM lanes 32 (w % 4) .. +31; lane = token row of the tile
-        const int quad = warp & 3;
-        float acc[kTcBN];
+        // epilogue warps: warp w may touch TMEM lanes 32 (w % 4) .. +31 (lane = token row of the tile);
+        // the two warps of a quadrant take 64 columns each, all their loads of a block in flight at once
+        const int quad = warp & 3, half = (warp - 2) >> 2;
+        float acc[kTcEpiCols];
 #pragma unroll
-        for (int i = 0; i < kTcBN; ++i) acc[i] = 0.f;
+        for (int i = 0; i < kTcEpiCols; ++i) acc[i] = 0.f;
         for (int kb = 0; kb < g.k_blocks; ++kb) {
             const int buf = kb & 1;
             mbar_wait(&tfull[buf], (kb >> 1) & 1, g.err, kErrTcAccum);
             tc_fence_after();
+            const uint32_t ta = tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kTcBN + half * kTcEpiCols;
+            uint32_t v0[32], v1[32];
+            tmem_ld32_issue(ta, v0);
+            tmem_ld32_issue(ta + 32, v1);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int cb = 0; cb < kTcBN / 32; ++cb) {
-                float v[32];
-                tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kTcBN + cb * 32, v);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) acc[cb * 32 + i] += v[i];
+            for (int i = 0; i < 32; ++i) {
+                acc[i] += __uint_as_float(v0[i]);
+                acc[32 + i] += __uint_as_float(v1[i]);
             }
             tc_fence_before();
             __syncwarp();
@@ -241,13 +242,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
         }
         const int row = m_tile * kTcBM + quad * 32 + lane;
         if (row < g.m_rows) {
-            const int n0 = n_tile * kTcBN;
+            const int n0 = n_tile * kTcBN + half * kTcEpiCols;
             if (g.mode == kTcSwigluSplit) {
                 uint16_t* ph = g.out_hi + (size_t)row * g.ld_hl + (n0 >> 1);
                 uint16_t* pm = g.out_mid + (size_t)row * g.ld_hl + (n0 >> 1);
                 uint16_t* pl = g.out_lo + (size_t)row * g.ld_hl + (n0 >> 1);
 #pragma unroll
-                for (int j = 0; j < kTcBN / 2; ++j) {
+                for (int j = 0; j < kTcEpiCols / 2; ++j) {
                     if (n0 + 2 * j + 1 < g.n_cols) {
                         const float gt = acc[2 * j], up = acc[2 * j + 1];
                         uint16_t hi, mid, lo;
@@ -260,7 +261,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
             } else {
                 float* po = g.out + (size_t)row * g.ldo + n0;
 #pragma unroll
-                for (int j = 0; j < kTcBN; ++j) {
+                for (int j = 0; j < kTcEpiCols; ++j) {
                     if (n0 + j < g.n_cols) po[j] = (g.mode == kTcResid) ? po[j] + acc[j] : acc[j];
                 }
             }
