@@ -61,6 +61,7 @@ struct Cfg {
 
 struct Prog {
     int mode, k, l, d, b, start, pos, la, n_seg_a, n_fused, embed_main, n_phases;
+    int n_main;   // fused attention phases: CTAs of the main row when the lanes get disjoint CTAs, else 0
 };
 
 struct OpDesc {            // one matrix product of a phase, as seen by this CTA
@@ -73,10 +74,17 @@ struct OpDesc {            // one matrix product of a phase, as seen by this CTA
 };
 
 struct AttnDesc {          // the attention items (head, KV page) of one lane in a phase, as seen by this CTA
-    // Items are numbered j = head * n_splits + page; CTA index c (after the lane's offset) owns the
-    // contiguous range [c*q, (c+1)*q), so its items belong to one head or two and are pre-merged
-    // inside the CTA; a head is covered by n_segs(head) consecutive CTAs.
+    // A CTA's work is a list of segments; a segment = consecutive pages of one head, folded and
+    // pre-merged inside the CTA.  Two ways of cutting the lane's items into segments:
+    //  - by head (short contexts, where latency rules): every head is cut into n_segs runs of q
+    //    pages; the (head, run) pairs are dealt round-robin to the lane's CTAs, normally one each;
+    //  - contiguous (long contexts, where the KV stream must be balanced): items are numbered
+    //    j = head * n_splits + page and CTA c owns [c*q, (c+1)*q) -- one head or two.
+    // The cut (scheme, q, n_segs) depends on the row's position and the grid only -- never on which
+    // lane the row is in or how many CTAs the lane got -- so a token's attention is the same
+    // arithmetic whether it runs as a branch row, as the main row beside branches, or alone.
     int M, p, n_splits, s_tail, total, q, j0, j1, c_idx;
+    int by_head, n_segs, n_lane;   // scheme, runs per head, CTAs of the lane
     bool chunk;            // prefill chunk: row m sits at position p + m and also sees the new tokens of rows < m
     const float* qkv;
     uint16_t* kv_layer;
@@ -108,10 +116,21 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// A row at position p is cut by head while a lane's items are few per CTA (7B on 148 SMs: up to
+// 704 positions); q pages per run such that a head has at most grid / H runs.
+__device__ __forceinline__ bool cut_by_head(int H, int p) {
+    const int G = gridDim.x;
+    return G >= 2 * H && 2 * H * (p / kPageTokens + 1) <= 5 * G;
+}
+__device__ __forceinline__ int by_head_q(int H, int n_splits) {
+    const int cph = max(1, min(n_splits, (int)gridDim.x / H));
+    return (n_splits + cph - 1) / cph;
+}
+
 __device__ Prog build_prog(const FusedArgs& a) {
     Prog P;
     P.mode = a.mode; P.k = a.k; P.l = a.l; P.d = a.d;
-    P.b = 0; P.start = 0;
+    P.b = 0; P.start = 0; P.n_main = 0;
     if (a.mode == kPrefillChunk) {
         // k consecutive prompt tokens as the k rows of the "branch" lane through all d layers; the main
         // lane is idle.  Rows sit at positions pos .. pos+k-1 and attend causally inside the chunk.
@@ -135,6 +154,21 @@ __device__ Prog build_prog(const FusedArgs& a) {
     P.embed_main = P.start == 0;
     P.n_phases = P.embed_main + 5 * P.n_seg_a + (a.mode == kPpdStep ? 2 + 5 * P.n_fused : 0) +
                  (a.mode != kPrefillToken ? 2 : 0) + 1;
+    if (a.mode == kPpdStep && cut_by_head(a.H, P.pos) && cut_by_head(a.H, P.pos + 1)) {
+        // Split of the grid between the main row and the k branch rows in a fused attention phase:
+        // a segment's time ~ (its (half page, row) units per warp) + a fixed part; each lane deals
+        // its H * n_segs segments round-robin to its CTAs; take the split with the shortest phase.
+        const int G = gridDim.x;
+        const int nm = P.pos / kPageTokens + 1, nb = (P.pos + 1) / kPageTokens + 1;
+        const int qm = by_head_q(a.H, nm), qb = by_head_q(a.H, nb);
+        const int sm = a.H * ((nm + qm - 1) / qm), sb = a.H * ((nb + qb - 1) / qb);
+        const int tm = 5 * ((2 * qm + kCW - 1) / kCW) + 3, tb = 5 * ((2 * qb * a.k + kCW - 1) / kCW) + 3;
+        int best = 0x7FFFFFFF;
+        for (int n = 1; n < G; ++n) {
+            const int cost = max(((sm + n - 1) / n) * tm, ((sb + G - n - 1) / (G - n)) * tb);
+            if (cost < best) { best = cost; P.n_main = n; }
+        }
+    }
     return P;
 }
 
@@ -206,16 +240,58 @@ __device__ void fill_op(const FusedArgs& a, int kind, int layer, const LaneBuf& 
     o.first_rg = ((int)blockIdx.x - cta_off + G) % G;
 }
 
-__device__ void fill_attn(const FusedArgs& a, int layer, const LaneBuf& ln, int M, int p, bool branch, int cta_off, AttnDesc& t) {
+struct Seg { int h, s_lo, s_hi, r, n_segs; };   // pages [s_lo, s_hi) of head h; run r of n_segs
+
+// i-th segment of this CTA in the lane; false when there is none
+__device__ __forceinline__ bool segment(const AttnDesc& t, int H, int i, Seg& sg) {
+    if (t.by_head) {
+        const int pr = t.c_idx + i * t.n_lane;            // (head, run) pair
+        if (t.c_idx >= t.n_lane || pr >= H * t.n_segs) return false;
+        sg.h = pr / t.n_segs;
+        sg.r = pr - sg.h * t.n_segs;
+        sg.s_lo = sg.r * t.q;
+        sg.s_hi = min(t.n_splits, sg.s_lo + t.q);
+        sg.n_segs = t.n_segs;
+        return true;
+    }
+    int j = t.j0;
+    for (int k = 0; j < t.j1; ++k) {
+        const int h = j / t.n_splits;
+        const int s_lo = j - h * t.n_splits;
+        const int s_hi = min(t.n_splits, s_lo + (t.j1 - j));
+        if (k == i) {
+            const int c_first = (h * t.n_splits) / t.q;
+            sg.h = h; sg.s_lo = s_lo; sg.s_hi = s_hi;
+            sg.n_segs = ((h + 1) * t.n_splits - 1) / t.q - c_first + 1;
+            sg.r = t.c_idx - c_first;
+            return true;
+        }
+        j += s_hi - s_lo;
+    }
+    return false;
+}
+
+// cta_off / n_lane: the lane's CTAs are cta_off, cta_off + 1, .. (mod grid), n_lane of them
+__device__ void fill_attn(const FusedArgs& a, int layer, const LaneBuf& ln, int M, int p, bool branch, int cta_off, int n_lane,
+                          AttnDesc& t) {
     const int G = gridDim.x;
     t.M = M; t.p = p;
     t.n_splits = p / kPageTokens + 1;
     t.s_tail = p / kPageTokens;
     t.total = a.H * t.n_splits;
-    t.q = (t.total + G - 1) / G;
     t.c_idx = ((int)blockIdx.x - cta_off + G) % G;
-    t.j0 = min(t.total, t.c_idx * t.q);
-    t.j1 = min(t.total, t.j0 + t.q);
+    t.n_lane = n_lane;
+    t.by_head = cut_by_head(a.H, p) ? 1 : 0;
+    if (t.by_head) {
+        t.q = by_head_q(a.H, t.n_splits);
+        t.n_segs = (t.n_splits + t.q - 1) / t.q;
+        t.j0 = t.j1 = 0;
+    } else {               // always over the whole grid (n_lane == G)
+        t.n_segs = 0;
+        t.q = (t.total + G - 1) / G;
+        t.j0 = min(t.total, t.c_idx * t.q);
+        t.j1 = min(t.total, t.j0 + t.q);
+    }
     t.chunk = a.mode == kPrefillChunk;
     t.qkv = ln.qkv;
     t.kv_layer = a.kv + (size_t)layer * a.kv_layer_elems;
@@ -235,10 +311,19 @@ __device__ void make_phase(const FusedArgs& a, const Prog& P, int ph, int MB, Ph
         pd.n_ops = 1;
         if (lb >= 0) { fill_op(a, pd.kind, lb, a.br, MB, chunk ? 0 : G / 2, pd.op[1]); pd.n_ops = 2; }
     } else if (pd.kind == PH_ATTN) {
-        if (lm >= 0) fill_attn(a, lm, a.main, 1, P.pos, false, 0, pd.at[0]);
-        else { AttnDesc& t = pd.at[0]; t.total = 0; t.j0 = t.j1 = 0; t.q = 1; t.n_splits = 1; t.M = 1; t.chunk = false; }
+        const int p_br = chunk ? P.pos : P.pos + 1;
+        // When both lanes are active and both are cut by head, they get disjoint CTAs (P.n_main for
+        // the main row, the rest for the branch rows); otherwise each lane spreads over the grid.
+        const bool both = lm >= 0 && lb >= 0;
+        const bool disjoint = both && P.n_main > 0;
+        if (lm >= 0) fill_attn(a, lm, a.main, 1, P.pos, false, 0, disjoint ? P.n_main : G, pd.at[0]);
+        else { AttnDesc& t = pd.at[0]; t.total = 0; t.j0 = t.j1 = 0; t.q = 1; t.n_splits = 1; t.M = 1; t.chunk = false; t.by_head = 0; t.n_segs = 0; t.n_lane = 1; t.c_idx = 0; }
         pd.n_ops = 1;
-        if (lb >= 0) { fill_attn(a, lb, a.br, MB, chunk ? P.pos : P.pos + 1, true, chunk ? 0 : G / 2, pd.at[1]); pd.n_ops = 2; }
+        if (lb >= 0) {
+            if (disjoint) fill_attn(a, lb, a.br, MB, p_br, true, P.n_main, G - P.n_main, pd.at[1]);
+            else fill_attn(a, lb, a.br, MB, p_br, true, (chunk || !both) ? 0 : G / 2, G, pd.at[1]);
+            pd.n_ops = 2;
+        }
     } else if (pd.kind == PH_HEAD_EARLY || pd.kind == PH_HEAD_FINAL) {
         OpDesc& o = pd.op[0];
         o.w = pd.kind == PH_HEAD_EARLY ? a.w_head_early : a.w_head; o.N = a.V; o.K = a.D; o.x = a.main.h; o.ldx = a.Dp; o.gain = a.g_final; o.resid = nullptr;
@@ -284,14 +369,17 @@ __device__ __forceinline__ void for_each_item(const FusedArgs& a, const Prog& P,
             for (int ln = 0; ln < pd.n_ops; ++ln) {
                 const AttnDesc& t = pd.at[ln];
                 it.lane = ln;
-                for (int j = t.j0; j < t.j1; ++j) {
-                    it.h = j / t.n_splits;
-                    it.s = j - it.h * t.n_splits;
-                    it.n_valid = min(kPageTokens, t.p - it.s * kPageTokens);
-                    it.tail = it.s == t.s_tail;
-                    // a branch row's prefix ends with the position the main pass wrote in this launch
-                    it.kv_late = P.mode == kPpdStep && ln == 1 && it.s == P.pos / kPageTokens;
-                    f(pd, it);
+                Seg sg;
+                for (int i = 0; segment(t, a.H, i, sg); ++i) {
+                    it.h = sg.h;
+                    for (int sp = sg.s_lo; sp < sg.s_hi; ++sp) {
+                        it.s = sp;
+                        it.n_valid = min(kPageTokens, t.p - it.s * kPageTokens);
+                        it.tail = it.s == t.s_tail;
+                        // a branch row's prefix ends with the position the main pass wrote in this launch
+                        it.kv_late = P.mode == kPpdStep && ln == 1 && it.s == P.pos / kPageTokens;
+                        f(pd, it);
+                    }
                 }
             }
         } else {
@@ -721,7 +809,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
     using C = Cfg<MB>;
     constexpr int DPL = HD / 32, HALF = HD / 2, REC = HD + 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = gridDim.x, H = a.H;
+    const int H = a.H;
     int* err = a.state + S_ERR;
     const float sscale = 1.4426950408889634f / sqrtf((float)HD);
     const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
@@ -732,20 +820,17 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
     const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
     // rotation of position p (every decode row sits there), fetched before the first stage arrives
     float2 cs_p[DPL];
-    if (t.j0 < t.j1) {
+    Seg sg;
+    if (segment(t, H, 0, sg)) {
 #pragma unroll
         for (int jj = 0; jj < DPL; ++jj) cs_p[jj] = __ldg(a.rope + (size_t)t.p * HALF + i0 + jj);
     }
-    for (int jseg = t.j0; jseg < t.j1;) {
-        // segment: this CTA's items of one head
-        const int h = jseg / t.n_splits;
-        const int s_lo = jseg - h * t.n_splits;
-        const int s_hi = min(t.n_splits, s_lo + (t.j1 - jseg));
-        jseg += s_hi - s_lo;
-        // CTAs covering this head, and this CTA's rank among them
-        const int c_first = (h * t.n_splits) / t.q;
-        const int n_segs = ((h + 1) * t.n_splits - 1) / t.q - c_first + 1;
-        const int r = t.c_idx - c_first;
+    for (int iseg = 0; segment(t, H, iseg, sg); ++iseg) {
+        // segment: this CTA's pages of one head; its run index among the CTAs covering the head
+        const int h = sg.h, s_lo = sg.s_lo, s_hi = sg.s_hi, n_segs = sg.n_segs, r = sg.r;
+        // rows of the same half page go to warps `stride` apart, so that a short segment still
+        // spreads its (half page, row) units over all warps
+        const int stride = min(kCW, 2 * (s_hi - s_lo));
         float run_mx[M], run_sum[M], run_o[M][DPL];
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -765,15 +850,18 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                 const uint16_t* ks = reinterpret_cast<const uint16_t*>(st);
                 const uint16_t* vs = ks + kPageTokens * HD;
                 const float* qraw = reinterpret_cast<const float*>(st + C::kXOff);
-#pragma unroll
+                // One copy of the unit's code for all halves and rows (the loops are not unrolled and the
+                // running states are indexed at run time): the code runs once or twice per phase, so its
+                // cost is instruction fetch, and every unrolled copy would be fetched cold.
+#pragma unroll 1
                 for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
+#pragma unroll 1
                     for (int m = 0; m < M; ++m) {
                         // Work unit = (half page, row): unit u = 2 * page + half of the segment, row m ->
-                        // warp (u + m) % 8, so the halves and rows of one page spread over the warps.  For
-                        // every row the units a warp folds together are those with the same u % 8,
-                        // whatever M is.
-                        if ((2 * (s - s_lo) + hf + m) % kCW != warp) continue;
+                        // warp (u + m * stride) % 8, so the halves and rows of one page spread over the
+                        // warps.  For every row the units a warp folds together are those with the same
+                        // u % 8, whatever M is.
+                        if ((2 * (s - s_lo) + hf + m * stride) % kCW != warp) continue;
                         const int nv = min(32, n_valid - 32 * hf);              // cached positions in this half
                         const bool has_new = tail && (n_valid >> 5) == hf;     // the new token falls into this half
                         if (nv <= 0 && !has_new) continue;
@@ -896,12 +984,12 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
         consumer_sync();
         for (int idx = tid; idx < M * HD; idx += kCW * 32) {
             const int m = idx / HD, jd = idx - m * HD;
-            // unit groups c = 0..7 (units u with u % 8 == c) in order; group c of row m sits in warp (c + m) % 8
-            const float* rec0 = ws + ((size_t)(m % kCW) * M + m) * REC;
+            // unit groups c = 0..7 (units u with u % 8 == c) in order; group c of row m sits in warp (c + m * stride) % 8
+            const float* rec0 = ws + ((size_t)((m * stride) % kCW) * M + m) * REC;
             float mx = rec0[HD], num = rec0[jd], den = rec0[HD + 1];
 #pragma unroll
             for (int c = 1; c < kCW; ++c) {
-                const float* rec = ws + ((size_t)((c + m) % kCW) * M + m) * REC;
+                const float* rec = ws + ((size_t)((c + m * stride) % kCW) * M + m) * REC;
                 const float ms = rec[HD];
                 const float nm = fmaxf(mx, ms);
                 const float wa = exp2f(mx - nm), wb = exp2f(ms - nm);
@@ -931,11 +1019,9 @@ __device__ void attn_merge(const FusedArgs& a, const AttnDesc& t, const Shared& 
     const int tid = threadIdx.x;
     const int H = a.H;
     float* stage = reinterpret_cast<float*>(sh.un + C::kMerge);
-    for (int jseg = t.j0; jseg < t.j1;) {
-        const int h = jseg / t.n_splits;
-        jseg = min(t.j1, (h + 1) * t.n_splits);
-        const int c_first = (h * t.n_splits) / t.q;
-        const int n_segs = ((h + 1) * t.n_splits - 1) / t.q - c_first + 1;
+    Seg sg;
+    for (int iseg = 0; segment(t, H, iseg, sg); ++iseg) {
+        const int h = sg.h, n_segs = sg.n_segs;
         if (n_segs == 1) continue;        // finished inside this CTA
         if (tid == 0) sh.flags[0] = atomicAdd(&t.tickets[h], 1) == n_segs - 1;
         consumer_sync();
