@@ -775,29 +775,13 @@ __device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh,
 __device__ __forceinline__ float rot_lo(float x0, float x1, float2 cs) { return __fmaf_rn(x0, cs.x, -__fmul_rn(x1, cs.y)); }
 __device__ __forceinline__ float rot_hi(float x0, float x1, float2 cs) { return __fmaf_rn(x1, cs.x, __fmul_rn(x0, cs.y)); }
 
-// Sum over the 32 lanes of 32 per-lane values at once: after the call lane t holds the total of
-// v[t].  31 shuffles instead of 160; the order of additions is a fixed butterfly.
-__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane) {
-#pragma unroll
-    for (int half = 16; half >= 1; half >>= 1) {
-        const bool upper = (lane & half) != 0;
-#pragma unroll
-        for (int i = 0; i < half; ++i) {
-            const float keep = upper ? v[i + half] : v[i];
-            const float send = upper ? v[i] : v[i + half];
-            v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, half);
-        }
-    }
-    return v[0];
-}
-
 // Attention of one lane: this CTA's contiguous range of (head, KV page) items, cut into segments
 // of one head.  K/V tiles and the raw q (and, for the page that receives the new token, the raw k
 // and v) rows arrive through the ring.
 //  - Each (half page of 32 positions, row) is processed by ONE warp, so a few pages already keep
-//    all eight warps busy: lane j owns dims [j*DPL, (j+1)*DPL) of the head; the 32 scores are
-//    reduced across lanes together (lane t ends up owning position t); softmax statistics by
-//    shuffles; P.V with the probabilities broadcast from their owner lanes.
+//    all eight warps busy: lane t computes the score of position t of the half page (q from a
+//    per-warp shared buffer); softmax statistics by shuffles; for P.V lane j owns dims
+//    [j*DPL, (j+1)*DPL) of the head and the probabilities are broadcast from their owner lanes.
 //  - A warp folds its units into a running (max, sum, P.V) per row in registers; the 8 warp states
 //    of a segment are merged through shared memory in a fixed group order.
 //  - A head covered by one CTA is finished there.  Otherwise every covering CTA writes one record
@@ -815,6 +799,7 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
     const size_t page_elems = (size_t)2 * H * kPageTokens * HD;
     const float NEG = __int_as_float(0xFF800000);
     float* ws = reinterpret_cast<float*>(sh.un + C::kWs);          // [warp][m][REC]
+    float* qs = reinterpret_cast<float*>(sh.un + C::kMerge) + (threadIdx.x >> 5) * HD;   // this warp's rotated q (the merge staging area is idle here)
     const int d0 = lane * DPL;
     const bool lo = d0 < HALF;
     const int i0 = lo ? d0 : d0 - HALF;       // index of this lane's rotate-half pairs
@@ -874,27 +859,29 @@ __device__ void attn_consume(const FusedArgs& a, const AttnDesc& t, const Shared
                             const float x0 = qraw[m * HD + i0 + jj], x1 = qraw[m * HD + i0 + jj + HALF];
                             qr[jj] = lo ? rot_lo(x0, x1, csq) : rot_hi(x0, x1, csq);
                         }
-                        // scores in log2 units: lane t gets position 32*hf + t; new tokens take lanes nv, nv+1, ..
+                        // Scores in log2 units: lane t computes position 32*hf + t itself, walking the head
+                        // dimension in chunks of 4 starting at chunk t (so the lanes of a half warp read
+                        // different banks of their K rows); the rotated q comes from this warp's shared
+                        // buffer.  Four accumulators (one per element of a chunk), added pairwise at the
+                        // end.  New tokens take lanes nv, nv+1, ..
+                        __syncwarp();
+#pragma unroll
+                        for (int jj = 0; jj < DPL; ++jj) qs[d0 + jj] = qr[jj];
+                        __syncwarp();
                         float sc = NEG;
                         if (nv > 0) {
-                            float part[32];
-#pragma unroll
-                            for (int tt = 0; tt < 32; ++tt) {
-                                const int pos = hf * 32 + tt;
-                                float kf[DPL];
-                                if constexpr (DPL == 4) {
-                                    const uint2 kk = *reinterpret_cast<const uint2*>(ks + pos * HD + lane * 4);
-                                    kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
-                                } else {
-                                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(ks + pos * HD + lane * 2);
-                                    kf[0] = bf16_lo(kk); kf[1] = bf16_hi(kk);
-                                }
-                                float dsum = 0.f;
-#pragma unroll
-                                for (int jj = 0; jj < DPL; ++jj) dsum = fmaf(qr[jj], kf[jj], dsum);
-                                part[tt] = dsum;       // rows >= nv hold stale bytes: masked below
+                            constexpr int NC = HD / 4;
+                            const uint16_t* krow = ks + (hf * 32 + lane) * HD;   // rows >= nv hold stale bytes: masked below
+                            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+                            for (int j = 0; j < NC; ++j) {
+                                const int c = (j + lane) & (NC - 1);
+                                const uint2 kk = *reinterpret_cast<const uint2*>(krow + c * 4);
+                                const float4 qq = *reinterpret_cast<const float4*>(qs + c * 4);
+                                a0 = fmaf(qq.x, bf16_lo(kk.x), a0); a1 = fmaf(qq.y, bf16_hi(kk.x), a1);
+                                a2 = fmaf(qq.z, bf16_lo(kk.y), a2); a3 = fmaf(qq.w, bf16_hi(kk.y), a3);
                             }
-                            const float tot = transpose_reduce32(part, lane) * sscale;
+                            const float tot = __fadd_rn(__fadd_rn(a0, a1), __fadd_rn(a2, a3)) * sscale;
                             sc = lane < nv ? tot : NEG;
                         }
                         const int nvp = nv > 0 ? nv : 0;
