@@ -177,6 +177,11 @@ int ppd_debug_phase_times(ppd_ctx* ctx, int32_t enable, uint64_t* out, int32_t n
  * 0..n_pages-1, n_pages = ceil(max_seq / kv_page_tokens)); only valid right after create or
  * before prefill.  Exists to test that kernels honour the page table. */
 int ppd_debug_set_page_table(ppd_ctx* ctx, const int32_t* table, int32_t n_pages);
+/* Number of CTAs the kernels are launched with (8 .. SM count of the device; 0 restores the SM
+ * count).  The way attention is cut into segments depends on the grid, so a small grid reaches, on
+ * a tiny model, the code paths a large model reaches on the full grid (several segments per CTA,
+ * the contiguous cut of long contexts).  Results differ in rounding only.  Between steps only. */
+int ppd_debug_set_grid(ppd_ctx* ctx, int32_t n_ctas);
 
 const char* ppd_strerror(int code);
 /* Text of the last CUDA error seen by this context (static storage). */

@@ -62,6 +62,7 @@ SIGNATURES = {
     "ppd_debug_logits": (ctypes.c_int, [_P, _P, _P]),
     "ppd_debug_last": (ctypes.c_int, [_P, _P, _P, _I]),
     "ppd_debug_force_token": (ctypes.c_int, [_P, _I]),
+    "ppd_debug_set_grid": (ctypes.c_int, [_P, _I]),
     "ppd_debug_set_page_table": (ctypes.c_int, [_P, _P, _I]),
     "ppd_debug_phase_times": (ctypes.c_int, [_P, _I, _P, _I]),
     "ppd_strerror": (ctypes.c_char_p, [ctypes.c_int]),
@@ -265,6 +266,11 @@ class Context:
             _check(self.lib.ppd_debug_phase_times(self._h, 1 if enable else 0,
                                                   out.ctypes.data if n_phases else None, n_phases), self._h)
         return out[:, :n_phases]
+
+    def set_grid(self, n_ctas):
+        """CTAs per launch (0 = one per SM); a small grid exercises the multi-segment attention paths."""
+        with self._dev():
+            _check(self.lib.ppd_debug_set_grid(self._h, n_ctas), self._h)
 
     def set_page_table(self, table):
         t = np.ascontiguousarray(table, dtype=np.int32)

@@ -948,6 +948,18 @@ int ppd_debug_set_page_table(ppd_ctx* x, const int32_t* table, int32_t n_pages) 
     return PPD_OK;
 }
 
+int ppd_debug_set_grid(ppd_ctx* x, int32_t n_ctas) {
+    if (!x || n_ctas < 0) return PPD_EINVAL;
+    int dev = 0, sms = 0;
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (n_ctas > sms || (n_ctas != 0 && n_ctas < kMaxRows)) return PPD_EINVAL;   // the embedding phases use one CTA per row
+    CK(cudaStreamSynchronize(x->sm));
+    CK(cudaStreamSynchronize(x->sb));
+    x->n_sms = n_ctas == 0 ? sms : n_ctas;
+    return PPD_OK;
+}
+
 const char* ppd_strerror(int code) {
     switch (code) {
         case PPD_OK: return "ok";

@@ -418,3 +418,25 @@ def test_tensor_core_prefill_7b_shapes_two_layers():
     ctx.set_prefill_chunk(0)
     check_against_oracle(shape, blob, prompt, 3, 3, 1, ctx=ctx, max_k=3)
     ctx.close()
+
+
+@pytest.mark.parametrize("grid,n_prompt", [(8, 100), (8, 300), (8, 400), (12, 330), (37, 200)])
+def test_small_grids_reach_the_other_attention_cuts(tiny_shape, tiny_blob, grid, n_prompt):
+    """The attention work split depends on the grid: on a few CTAs the tiny model goes through what
+    a large model meets on the full grid -- several segments per CTA, lanes sharing CTAs, and (8
+    CTAs beyond 320 positions) the contiguous cut of long contexts.  Same checks as on the full grid."""
+    prompt = ppd_inputs.gen_prompt(tiny_shape.vocab, n_prompt, seed=41)
+    ctx = ppd.Context(tiny_shape, max_seq=n_prompt + 60, max_k=5)
+    ctx.load_weights(tiny_blob)
+    ctx.set_grid(grid)
+    check_against_oracle(tiny_shape, tiny_blob, prompt, 8, 3, 2, ctx=ctx, max_k=5)
+    ctx.prefill(prompt)
+    g, _, gfl, _, _ = gpu_stream(ctx, 0, 0, 40)
+    for k, l in ((3, 2), (5, 1), (2, 3)):
+        ctx.prefill(prompt)
+        p, _, pfl, _, _ = gpu_stream(ctx, k, l, 40)
+        assert (p == g).all() and np.array_equal(pfl, gfl), (k, l)
+    with pytest.raises(ppd.PPDError):
+        ctx.set_grid(3)
+    ctx.set_grid(0)
+    ctx.close()
