@@ -1066,6 +1066,32 @@ __device__ void run_attn_merge(const FusedArgs& a, const AttnDesc& t, const Shar
     else attn_merge<M, 64, MB>(a, t, sh);
 }
 
+// One row of the embedding table (bf16) to float.  The row is almost never in L2, so all of a
+// thread's 16-byte loads are issued before the first use: one HBM round trip, not D / 256 of them.
+__device__ __forceinline__ void embed_row(const uint16_t* e, float* h, int D, int tid) {
+    if ((D & 7) == 0 && D <= 8 * 4 * kCW * 32) {
+        const uint4* src = reinterpret_cast<const uint4*>(e);
+        const int n = D >> 3;
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = tid + j * kCW * 32;
+            v[j] = i < n ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = tid + j * kCW * 32;
+            if (i < n) {
+                float4* dst = reinterpret_cast<float4*>(h + (size_t)i * 8);
+                dst[0] = make_float4(bf16_lo(v[j].x), bf16_hi(v[j].x), bf16_lo(v[j].y), bf16_hi(v[j].y));
+                dst[1] = make_float4(bf16_lo(v[j].z), bf16_hi(v[j].z), bf16_lo(v[j].w), bf16_hi(v[j].w));
+            }
+        }
+    } else {
+        for (int i = tid; i < D; i += kCW * 32) h[i] = bf16_bits_to_f32(e[i]);
+    }
+}
+
 // verify + commit (Algorithm 2): on a match the branch's K/V of layers 1..b go to cache position
 // pos+1 and its hidden state becomes the main one.  CTA c copies layers c, c+G, ...
 __device__ void commit_copy(const FusedArgs& a, const Prog& P) {
@@ -1168,15 +1194,13 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
             case PH_EMBED_MAIN:
                 if (blockIdx.x == 0) {
                     const int tok = a.mode == kPrefillToken ? __ldcg(a.token_src) : __ldcg(a.state + S_PENDING);
-                    const uint16_t* e = a.emb + (size_t)tok * a.D;
-                    for (int i = tid; i < a.D; i += kCW * 32) a.main.h[i] = bf16_bits_to_f32(e[i]);
+                    embed_row(a.emb + (size_t)tok * a.D, a.main.h, a.D, tid);
                 }
                 break;
             case PH_EMBED_BR:
                 if ((int)blockIdx.x < P.k) {
                     const int tok = P.mode == kPrefillChunk ? __ldcg(a.token_src + blockIdx.x) : __ldcg(a.top_early + blockIdx.x);
-                    const uint16_t* e = a.emb + (size_t)tok * a.D;
-                    for (int i = tid; i < a.D; i += kCW * 32) a.br.h[(size_t)blockIdx.x * a.Dp + i] = bf16_bits_to_f32(e[i]);
+                    embed_row(a.emb + (size_t)tok * a.D, a.br.h + (size_t)blockIdx.x * a.Dp, a.D, tid);
                 }
                 break;
             case PH_QKV: case PH_O: case PH_GU: case PH_DOWN:
