@@ -46,6 +46,15 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a library GEMM timed alone on this machine (burst figure)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 # ------------------------------------------------------------------ algorithmic bytes / flops
 
 def layer_bytes(s):
@@ -336,7 +345,12 @@ def run_gpu(args, wl):
         "speedup_vs_greedy": greedy_tok_ms / ppd_tok_ms,
         "prefill": {"ms": prefill_ms, "tokens": P - 1, "path": "tcgen05 GEMM + causal attention kernel",
                     # 2 flops per weight per prompt token = one flop per weight byte; the three-term split triples the MMA work
-                    "tflops_useful": s.n_layers * layer_bytes(s) * (P - 1) / (prefill_ms * 1e9)},
+                    "tflops_useful": s.n_layers * layer_bytes(s) * (P - 1) / (prefill_ms * 1e9),
+                    "roofline": {"bound": "tensor", "unit": "TFLOP/s", "peak": measured_tensor_peak()[0],
+                                 "peak_kind": measured_tensor_peak()[1],
+                                 "achieved_issued": 3.0 * s.n_layers * layer_bytes(s) * (P - 1) / (prefill_ms * 1e9),
+                                 "frac_issued": 3.0 * s.n_layers * layer_bytes(s) * (P - 1) / (prefill_ms * 1e9) / measured_tensor_peak()[0],
+                                 "note": "whole prompt pass incl. attention and elementwise kernels; bf16 MMA flops issued = 3 x useful"}},
         "p_correct": p_hat, "ppd_equals_greedy": exact,
         "ms_step_after_miss": t_fresh, "ms_step_after_hit": t_cont,
         "predicted_ms_per_token_p_correct_model": pred_ms,

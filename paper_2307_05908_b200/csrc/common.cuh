@@ -88,11 +88,6 @@ __device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gmem_src, u
         : "memory");
 }
 
-// Asks L2 to fetch [p, p + bytes) from HBM without bringing it to the SM (fire and forget).
-__device__ __forceinline__ void bulk_prefetch_l2(const void* gmem_src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gmem_src), "r"(bytes) : "memory");
-}
-
 // ---- programmatic dependent launch
 // wait: blocks until the kernels this launch depends on have completed and their writes are
 // visible (no-op for a normal launch).  launch_dependents: lets the next kernel in the stream

@@ -165,26 +165,13 @@ cudaError_t launch_commit(const CommitArgs& a, cudaStream_t st, bool pdl) {
     return cudaLaunchKernelEx(&cfg, commit_kernel, a);
 }
 
-// sets the small device state block
-__global__ void set_state_kernel(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step) {
-    if (threadIdx.x == 0) {
-        if (d_pos) *d_pos = pos;
-        if (d_pending) *d_pending = pending;
-        if (d_step) *d_step = step;
-    }
-}
-
+// sets words of the small device state block
 __global__ void write_words_kernel(int* base, WordWrites w) {
     if (threadIdx.x < w.n) base[w.idx[threadIdx.x]] = w.val[threadIdx.x];
 }
 
 cudaError_t launch_write_words(int* base, const WordWrites& w, cudaStream_t st) {
     write_words_kernel<<<1, 32, 0, st>>>(base, w);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_set_state(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step, cudaStream_t st) {
-    set_state_kernel<<<1, 32, 0, st>>>(d_pos, pos, d_pending, pending, d_step, step);
     return cudaGetLastError();
 }
 

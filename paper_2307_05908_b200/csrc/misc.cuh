@@ -43,6 +43,5 @@ cudaError_t launch_rope_table(float2* table, int n_pos, int hd, double theta, cu
 cudaError_t launch_commit(const CommitArgs& a, cudaStream_t st, bool pdl);
 struct WordWrites { int n; int idx[8]; int val[8]; };   // base[idx[i]] = val[i]
 cudaError_t launch_write_words(int* base, const WordWrites& w, cudaStream_t st);
-cudaError_t launch_set_state(int* d_pos, int pos, int* d_pending, int pending, int* d_step, int step, cudaStream_t st);
 
 }  // namespace ppd
