@@ -1,4 +1,4 @@
-"""Host-side logic of bench.py: byte/flop accounting against the survey's figures, and the
+"""Host-side logic of bench.py: byte/flop accounting against parameter counts worked out by hand, and the
 multi-rank plumbing (replicas, max over ranks) on two gloo ranks."""
 import json
 import os
