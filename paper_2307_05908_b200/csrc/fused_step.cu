@@ -111,10 +111,10 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // A row at position p is cut by head while a lane's items are few per CTA (7B on 148 SMs: up to
-// 704 positions); q pages per run such that a head has at most grid / H runs.
+// 1024 positions); q pages per run such that a head has at most grid / H runs.
 __device__ __forceinline__ bool cut_by_head(int H, int p) {
     const int G = gridDim.x;
-    return G >= 2 * H && 2 * H * (p / kPageTokens + 1) <= 5 * G;
+    return G >= 2 * H && 2 * H * (p / kPageTokens + 1) <= 7 * G;
 }
 __device__ __forceinline__ int by_head_q(int H, int n_splits) {
     const int cph = max(1, min(n_splits, (int)gridDim.x / H));
