@@ -197,7 +197,8 @@ def run_reference(args, wl):
 
 def workload_name(args, wl):
     return (f"{wl.shape.name}-shaped random-init bf16 (d={wl.shape.n_layers}, D={wl.shape.d_model}, F={wl.shape.d_ffn}, "
-            f"V={wl.shape.vocab}), prompt {args.prompt}, PPD k={args.k} at layer {args.l}, batch 1")
+            f"V={wl.shape.vocab}), prompt {args.prompt}, PPD k={args.k} at layer {args.l}, batch 1"
+            + (f", residual-branch init scale {args.resid_scale}" if getattr(args, "resid_scale", None) is not None else ""))
 
 
 # ------------------------------------------------------------------ GPU leg
@@ -248,7 +249,8 @@ def run_gpu(args, wl):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     s, k, l, K, W, P = wl.shape, args.k, args.l, args.steps, args.warmup, args.prompt
-    blob = ppd_inputs.gen_weights(s, seed=0)
+    blob = (ppd_inputs.gen_weights(s, seed=0) if args.resid_scale is None
+            else ppd_inputs.gen_weights(s, seed=0, resid_scale=args.resid_scale))
     prompt = ppd_inputs.gen_prompt(s.vocab, P, seed=1)
     ctx = ppd.Context(s, max_seq=P + W + K + 8, max_k=max(k, 1), device=f"cuda:{local}")
     ctx.load_weights(blob)
@@ -400,6 +402,9 @@ def main():
     ap.add_argument("--l", type=int, default=None)
     ap.add_argument("--prompt", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--resid-scale", type=float, default=None,
+                    help="scale of the residual-branch output matrices in the random init (default 0.1); smaller "
+                         "values raise the early head's hit rate: a knob to check the latency model across p_correct")
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the model to this many layers (small case for profiler captures)")
     args = ap.parse_args()
