@@ -224,6 +224,18 @@ size_t ppd_op_gemm_scratch_bytes(int32_t M, int32_t K);
 int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
                 float* out, int32_t ldo, void* scratch, size_t scratch_bytes, void* stream);
 
+/* The skinny product y[m][n] = sum_k W[n][k] x'[m][k] (x' = RMSNorm(x) if gain is given) for
+ * M <= 8 rows on the tensor cores, with the roles swapped: the packed weight tile is the 128-row
+ * operand of tcgen05.mma and the activation rows (three bf16 terms each) a 16-wide one, so the time
+ * does not depend on M.  Experimental building block (not used by ppd_decode yet): it shows what
+ * the k branch rows of Algorithm 2 would cost once the products leave the FMA pipe.
+ * scratch: device, 256-byte aligned, >= ppd_op_gemv_tc_scratch_bytes(K).  Asynchronous on stream;
+ * bounded device waits record a code in the first word of scratch. */
+size_t ppd_op_gemv_tc_scratch_bytes(int32_t K);
+int ppd_op_gemv_tc(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
+                   const float* gain, float eps, float* out, int32_t ldo, void* scratch,
+                   size_t scratch_bytes, void* stream);
+
 /* Head: logits[m][v] = W_H . RMSNorm(x[m]) for M rows and the k largest per row in the order
  * (value descending, id ascending).  scratch: device, >= ppd_op_head_scratch_bytes() bytes,
  * zeroed once by the caller before first use (the kernel leaves it zeroed).

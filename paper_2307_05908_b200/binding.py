@@ -72,6 +72,8 @@ SIGNATURES = {
     "ppd_op_gemv": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _I, _P]),
     "ppd_op_gemm_scratch_bytes": (_SZ, [_I, _I]),
     "ppd_op_gemm": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _I, _P, _SZ, _P]),
+    "ppd_op_gemv_tc_scratch_bytes": (_SZ, [_I]),
+    "ppd_op_gemv_tc": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _P, _I, _P, _SZ, _P]),
     "ppd_op_head_scratch_bytes": (_SZ, []),
     "ppd_op_head_topk": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P, _P]),
     "ppd_op_head_topk_static": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _P, _P]),
@@ -310,6 +312,18 @@ def op_gemm(w_packed, N, K, x, out, scratch, stream=None):
     M, ldx = x.shape
     _check(load().ppd_op_gemm(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx, out.data_ptr(), out.shape[1],
                               scratch.data_ptr(), scratch.numel() * scratch.element_size(), _s(stream)))
+
+
+def op_gemv_tc_scratch_bytes(K):
+    return load().ppd_op_gemv_tc_scratch_bytes(K)
+
+
+def op_gemv_tc(w_packed, N, K, x, gain, eps, out, scratch, stream=None):
+    """Skinny product (M <= 8 rows) with the weight tile as the wide tensor-core operand."""
+    M, ldx = x.shape
+    _check(load().ppd_op_gemv_tc(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx,
+                                 None if gain is None else gain.data_ptr(), eps, out.data_ptr(), out.shape[1],
+                                 scratch.data_ptr(), scratch.numel() * scratch.element_size(), _s(stream)))
 
 
 def op_head_topk(w_packed, vocab, K, x, gain, eps, k, scratch, logits, top_ids, top_vals, stream=None):

@@ -1042,6 +1042,35 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
     return h_err ? PPD_ETIMEOUT : PPD_OK;
 }
 
+size_t ppd_op_gemv_tc_scratch_bytes(int32_t K) {
+    if (K < 1) return 0;
+    return (size_t)3 * 8 * round_up(K, kTileCols) * 2 + 256;
+}
+
+int ppd_op_gemv_tc(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, const float* gain,
+                   float eps, float* out, int32_t ldo, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!w_packed || !x || !out || !scratch || N < 1 || K < 1 || M < 1 || M > 8 || ldx < K || ldo < N) return PPD_EINVAL;
+    if (((uintptr_t)scratch % kAlign) != 0) return PPD_EINVAL;
+    if (scratch_bytes < ppd_op_gemv_tc_scratch_bytes(K)) return PPD_ENOSPC;
+    if (tc_init() != 0) return PPD_ECUDA;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int Kp = (int)round_up(K, kTileCols);
+    int* err = reinterpret_cast<int*>(scratch);
+    uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256);
+    uint16_t* mid = hi + (size_t)8 * Kp;
+    uint16_t* lo = mid + (size_t)8 * Kp;
+    CKOP(cudaMemsetAsync(scratch, 0, ppd_op_gemv_tc_scratch_bytes(K), st));
+    CKOP(launch_pf_norm_split(x, ldx, gain, eps, M, K, hi, mid, lo, Kp, st));
+    CUtensorMap mw, ma, mm, mb;
+    if (tc_map_packed(&mw, reinterpret_cast<const uint16_t*>(w_packed), N, K) || tc_map_rows(&ma, hi, 8, Kp, 8) ||
+        tc_map_rows(&mm, mid, 8, Kp, 8) || tc_map_rows(&mb, lo, 8, Kp, 8))
+        return PPD_ECUDA;
+    TcGemvArgs g{};
+    g.m_rows = M; g.n_rows = N; g.k_blocks = (K + kTcBK - 1) / kTcBK; g.out = out; g.ldo = ldo; g.err = err;
+    CKOP(launch_tc_gemv(mw, ma, mm, mb, g, sm_count(), st));
+    return PPD_OK;
+}
+
 size_t ppd_op_head_scratch_bytes(void) { return kHeadScratchBytes + 2 * kMaxRows * 8 * 4; }
 
 int ppd_op_head_topk(const void* w_packed, int32_t vocab, int32_t K, const float* x, int32_t M, int32_t ldx,

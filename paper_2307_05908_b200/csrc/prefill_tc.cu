@@ -33,11 +33,11 @@ int tc_init() {
     return 0;
 }
 
-int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols) {
-    if (!g_encode || cols % kTcBK != 0) return -1;
+int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols, int box_rows) {
+    if (!g_encode || cols % kTcBK != 0 || box_rows < 1 || box_rows > 256) return -1;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)kTcBM};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)box_rows};
     const cuuint32_t es[2] = {1, 1};
     return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(base), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -98,13 +98,16 @@ __device__ __forceinline__ uint64_t sw128_desc(uint32_t saddr) {
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128.
 constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+__device__ __forceinline__ void umma_bf16_desc(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(da), "l"(db), "r"(kTcIdesc), "r"(accumulate)
+        "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    umma_bf16_desc(tmem_d, da, db, kTcIdesc, accumulate);
 }
 
 // arrives on the mbarrier once every matrix instruction issued so far by this thread has completed
@@ -125,6 +128,17 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// 16 consecutive accumulator columns of this thread's TMEM lane; the caller waits (tcgen05.wait::ld)
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }
@@ -271,6 +285,143 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kTcTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------ skinny product on the tensor cores
+//
+// y[m][n] = sum_k W[n][k] x[m][k] for up to 8 rows m, with the roles swapped: the packed WEIGHT tile
+// is the A operand (M = 128 weight rows), the activation rows are a narrow B operand (N = 16, rows
+// 8..15 zero), so the tensor pipe needs ~100 cycles per 16 KB of weights whatever the number of
+// rows, and the kernel is a pure stream over the weights.  Persistent: CTA c walks the 128-row
+// weight tiles c, c + grid, ..; the 64-column blocks of all its tiles form one pipeline (8 stages).
+// Exactness and accumulation as in the prompt GEMM: three bf16 terms per activation, one 64-column
+// block per TMEM buffer, promoted to fp32 registers by the epilogue warps.
+
+constexpr int kGvStages = 8;
+constexpr int kGvXRows = 8;                               // activation rows fetched per block
+constexpr int kGvN = 16;                                  // N of the matrix instruction
+constexpr int kGvXTile = kGvN * kTcBK * 2;                // 2 KB: 16 rows x 128 bytes (two swizzle atoms)
+constexpr int kGvStageBytes = kTcTile + 3 * kGvXTile;     // W | x_hi | x_mid | x_lo = 22 KB
+constexpr int kGvStageTx = kTcTile + 3 * kGvXRows * kTcBK * 2;
+constexpr int kGvThreads = 192;                           // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..5: epilogue
+constexpr int kGvTmemCols = 32;                           // two buffers of 16 columns
+constexpr int kGvSmem = kGvStages * kGvStageBytes + 1024 + 256;
+constexpr uint32_t kGvIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGvN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+
+__global__ void __launch_bounds__(kGvThreads, 1)
+tc_gemv_kernel(const __grid_constant__ CUtensorMap tW, const __grid_constant__ CUtensorMap tX_hi,
+               const __grid_constant__ CUtensorMap tX_mid, const __grid_constant__ CUtensorMap tX_lo, const TcGemvArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kGvStages * kGvStageBytes);
+    uint64_t* empty = full + kGvStages;
+    uint64_t* tfull = empty + kGvStages;
+    uint64_t* tempty = tfull + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGvStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&tfull[b], 1);
+            mbar_init(&tempty[b], 4);
+        }
+        fence_barrier_init();
+    }
+    // rows 8..15 of every activation tile (the second swizzle atom) are never fetched: zero them once
+    for (int i = threadIdx.x; i < kGvStages * 3 * (kGvXTile / 2 / 16); i += kGvThreads) {
+        const int tile = i / (kGvXTile / 2 / 16), off = i % (kGvXTile / 2 / 16);
+        const int s = tile / 3, term = tile % 3;
+        reinterpret_cast<uint4*>(smem + s * kGvStageBytes + kTcTile + term * kGvXTile + kGvXTile / 2)[off] = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kGvTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+                for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
+                    const int s = it % kGvStages;
+                    if (it >= kGvStages) mbar_wait(&empty[s], ((it / kGvStages) - 1) & 1, g.err, kErrTcEmpty);
+                    uint8_t* st = smem + s * kGvStageBytes;
+                    mbar_arrive_expect_tx(&full[s], kGvStageTx);
+                    tma_load_4d(st, &tW, (kb % 4) * kTcBK, 0, kb / 4, t * (kTcBM / kTileRows), &full[s]);
+                    tma_load_2d(st + kTcTile, &tX_hi, kb * kTcBK, 0, &full[s]);
+                    tma_load_2d(st + kTcTile + kGvXTile, &tX_mid, kb * kTcBK, 0, &full[s]);
+                    tma_load_2d(st + kTcTile + 2 * kGvXTile, &tX_lo, kb * kTcBK, 0, &full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int it = 0;
+            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+                for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
+                    const int s = it % kGvStages, buf = it & 1;
+                    if (it >= 2) mbar_wait(&tempty[buf], ((it >> 1) - 1) & 1, g.err, kErrTcAccum);
+                    mbar_wait(&full[s], (it / kGvStages) & 1, g.err, kErrTcFull);
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + s * kGvStageBytes);
+                    const uint32_t td = tmem_d + buf * kGvN;
+#pragma unroll
+                    for (int k4 = 0; k4 < kTcBK / 16; ++k4) {
+                        const uint64_t da = sw128_desc(sa + k4 * 32);
+#pragma unroll
+                        for (int term = 0; term < 3; ++term)
+                            umma_bf16_desc(td, da, sw128_desc(sa + kTcTile + term * kGvXTile + k4 * 32), kGvIdesc, (k4 | term) != 0);
+                    }
+                    umma_commit(&empty[s]);
+                    umma_commit(&tfull[buf]);
+                }
+            }
+        }
+    } else {
+        const int quad = warp & 3;      // TMEM lanes 32 quad .. +31 = weight rows of the tile
+        int it = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+            float acc[kGvN];
+#pragma unroll
+            for (int i = 0; i < kGvN; ++i) acc[i] = 0.f;
+            for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
+                const int buf = it & 1;
+                mbar_wait(&tfull[buf], (it >> 1) & 1, g.err, kErrTcAccum);
+                tc_fence_after();
+                uint32_t v[16];
+                tmem_ld16_issue(tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kGvN, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < kGvN; ++i) acc[i] += __uint_as_float(v[i]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[buf]);
+            }
+            const int n = t * kTcBM + quad * 32 + lane;
+            if (n < g.n_rows) {
+#pragma unroll
+                for (int m = 0; m < kGvXRows; ++m)
+                    if (m < g.m_rows) g.out[(size_t)m * g.ldo + n] = acc[m];
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kGvTmemCols) : "memory");
     }
 }
 
@@ -444,6 +595,20 @@ cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_mid, co
     if (g.m_rows < 1 || g.n_cols < 1 || g.k_blocks < 1) return cudaErrorInvalidValue;
     const int m_tiles = (g.m_rows + kTcBM - 1) / kTcBM, n_tiles = (g.n_cols + kTcBN - 1) / kTcBN;
     tc_gemm_kernel<<<m_tiles * n_tiles, kTcThreads, kTcSmem, st>>>(a_hi, a_mid, a_lo, w, g);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tc_gemv(const CUtensorMap& w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
+                           const TcGemvArgs& g, int n_ctas, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGvSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (g.m_rows < 1 || g.m_rows > kGvXRows || g.n_rows < 1 || g.k_blocks < 1 || n_ctas < 1) return cudaErrorInvalidValue;
+    const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
+    tc_gemv_kernel<<<n_ctas < n_tiles ? n_ctas : n_tiles, kGvThreads, kGvSmem, st>>>(w, x_hi, x_mid, x_lo, g);
     return cudaGetLastError();
 }
 

@@ -32,8 +32,8 @@ struct TcGemmArgs {
 
 // Resolves the driver's tensor-map encoder through the runtime (no link against the driver library).
 int tc_init();
-// 2-D map over row-major bf16 [rows][cols] (cols a multiple of 64), box 64 x 128, 128-byte swizzle.
-int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols);
+// 2-D map over row-major bf16 [rows][cols] (cols a multiple of 64), box 64 x box_rows, 128-byte swizzle.
+int tc_map_rows(CUtensorMap* map, const uint16_t* base, int rows, int cols, int box_rows = kTcBM);
 // 4-D map over a packed weight matrix ([row group][column chunk][32][256]), box = 64 columns of
 // four consecutive row groups: 128 weight rows x 128 bytes, 128-byte swizzle.
 int tc_map_packed(CUtensorMap* map, const uint16_t* packed, int n_rows, int n_cols);
@@ -41,6 +41,19 @@ int tc_map_packed(CUtensorMap* map, const uint16_t* packed, int n_rows, int n_co
 // C[m][n] = sum_k (A_hi + A_mid + A_lo)[m][k] * W[n][k], fp32 accumulation in tensor memory.
 cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_mid, const CUtensorMap& a_lo, const CUtensorMap& w,
                            const TcGemmArgs& g, cudaStream_t st);
+
+struct TcGemvArgs {
+    int m_rows;              // activation rows (<= 8)
+    int n_rows;              // weight rows N
+    int k_blocks;            // ceil(K / 64)
+    float* out;              // y[m][n]
+    long long ldo;
+    int* err;
+};
+// Skinny product on the tensor cores: the weight tile is the A operand, the (<= 8) activation rows,
+// as three bf16 terms each ([8][K] row-major, maps with box_rows = 8), are a narrow B operand.
+cudaError_t launch_tc_gemv(const CUtensorMap& w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
+                           const TcGemvArgs& g, int n_ctas, cudaStream_t st);
 
 // h[r][:] = E[tokens[r]][:]
 cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int D, float* h, int ldh, cudaStream_t st);

@@ -238,3 +238,36 @@ def test_tensor_core_gemm_against_oracle(N, K, M):
         ref = oracle.matvec(w, x[m].astype(np.float64))
         scale = np.abs(ref).max() + 1e-6
         assert np.abs(got[m, :N] - ref).max() < 3e-5 * scale + 1e-6, m
+
+
+@pytest.mark.parametrize("N,K", [(768, 256), (1000, 512), (96, 688), (2048, 11008)])
+@pytest.mark.parametrize("M", [1, 3, 8])
+def test_tensor_core_skinny_product(N, K, M):
+    """The skinny product with the weight tile as the wide tensor-core operand, against the oracle,
+    with and without the fused RMSNorm; a row's result must not depend on the rows beside it."""
+    rng = np.random.default_rng(N * 7 + K + M)
+    w = bf16_bits(rng, (N, K), 0.05)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    g = bf16_bits(rng, (K,), 1.0)
+    wp = pack(w)
+    xd = torch.from_numpy(x).to(DEV)
+    gd = torch.from_numpy(ppd_inputs.bf16_to_f32(g).astype(np.float32)).to(DEV)
+    scratch = torch.empty(ppd.op_gemv_tc_scratch_bytes(K), dtype=torch.uint8, device=DEV)
+    for gain in (None, gd):
+        out = torch.full((M, N + 3), 7.0, dtype=torch.float32, device=DEV)
+        ppd.op_gemv_tc(wp, N, K, xd, gain, 1e-5, out, scratch)
+        torch.cuda.synchronize()
+        assert int(scratch[:4].view(torch.int32).item()) == 0          # no bounded wait gave up
+        got = out.cpu().numpy()
+        assert (got[:, N:] == 7.0).all()
+        for m in range(M):
+            xin = x[m].astype(np.float64)
+            if gain is not None:
+                xin = oracle.rmsnorm(xin, g, 1e-5)
+            ref = oracle.matvec(w, xin)
+            scale = np.abs(ref).max() + 1e-6
+            assert np.abs(got[m, :N] - ref).max() < 2e-5 * scale + 1e-6, (m, gain is not None)
+        if M > 1:      # batch invariance: row 0 alone gives the same bits
+            out1 = torch.zeros((1, N + 3), dtype=torch.float32, device=DEV)
+            ppd.op_gemv_tc(wp, N, K, xd[:1].contiguous(), gain, 1e-5, out1, scratch)
+            assert np.array_equal(out1.cpu().numpy()[0, :N], got[0, :N])
