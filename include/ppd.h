@@ -229,10 +229,16 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
  * operand of tcgen05.mma and the activation rows (three bf16 terms each) a 16-wide one, so the time
  * does not depend on M.  Experimental building block (not used by ppd_decode yet): it shows what
  * the k branch rows of Algorithm 2 would cost once the products leave the FMA pipe.
+ * w_tc: device, the weights in the packing of ppd_op_pack_tc: 16 KB blocks of 128 rows x 64 columns,
+ * each stored as the operand sits in shared memory, so the kernel streams them with plain bulk
+ * copies (src of ppd_op_pack_tc: device, row-major bf16 [n_rows][n_cols]; dst: device, 16-byte
+ * aligned, ppd_op_tc_packed_bytes(n_rows, n_cols) bytes).
  * scratch: device, 256-byte aligned, >= ppd_op_gemv_tc_scratch_bytes(K).  Asynchronous on stream;
  * bounded device waits record a code in the first word of scratch. */
+size_t ppd_op_tc_packed_bytes(int32_t n_rows, int32_t n_cols);
+int ppd_op_pack_tc(const uint16_t* src, int32_t n_rows, int32_t n_cols, void* dst, void* stream);
 size_t ppd_op_gemv_tc_scratch_bytes(int32_t K);
-int ppd_op_gemv_tc(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
+int ppd_op_gemv_tc(const void* w_tc, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx,
                    const float* gain, float eps, float* out, int32_t ldo, void* scratch,
                    size_t scratch_bytes, void* stream);
 

@@ -72,6 +72,8 @@ SIGNATURES = {
     "ppd_op_gemv": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _I, _P, _P, _I, _P]),
     "ppd_op_gemm_scratch_bytes": (_SZ, [_I, _I]),
     "ppd_op_gemm": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _I, _P, _SZ, _P]),
+    "ppd_op_tc_packed_bytes": (_SZ, [_I, _I]),
+    "ppd_op_pack_tc": (ctypes.c_int, [_P, _I, _I, _P, _P]),
     "ppd_op_gemv_tc_scratch_bytes": (_SZ, [_I]),
     "ppd_op_gemv_tc": (ctypes.c_int, [_P, _I, _I, _P, _I, _I, _P, _F, _P, _I, _P, _SZ, _P]),
     "ppd_op_head_scratch_bytes": (_SZ, []),
@@ -312,6 +314,16 @@ def op_gemm(w_packed, N, K, x, out, scratch, stream=None):
     M, ldx = x.shape
     _check(load().ppd_op_gemm(w_packed.data_ptr(), N, K, x.data_ptr(), M, ldx, out.data_ptr(), out.shape[1],
                               scratch.data_ptr(), scratch.numel() * scratch.element_size(), _s(stream)))
+
+
+def op_pack_tc(src_bf16, dst=None, stream=None):
+    """Packs a row-major bf16 (int16 view) device matrix for op_gemv_tc; returns the packed buffer."""
+    import torch
+    n, k = src_bf16.shape
+    if dst is None:
+        dst = torch.empty(load().ppd_op_tc_packed_bytes(n, k), dtype=torch.uint8, device=src_bf16.device)
+    _check(load().ppd_op_pack_tc(src_bf16.data_ptr(), n, k, dst.data_ptr(), _s(stream)))
+    return dst
 
 
 def op_gemv_tc_scratch_bytes(K):

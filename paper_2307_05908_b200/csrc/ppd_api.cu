@@ -1044,13 +1044,26 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
 
 size_t ppd_op_gemv_tc_scratch_bytes(int32_t K) {
     if (K < 1) return 0;
-    return (size_t)3 * 8 * round_up(K, kTileCols) * 2 + 256;
+    return (size_t)3 * 8 * round_up(K, kTileCols) * 2 + 256 + kTcGemvPartialBytes;
 }
 
-int ppd_op_gemv_tc(const void* w_packed, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, const float* gain,
+size_t ppd_op_tc_packed_bytes(int32_t n_rows, int32_t n_cols) {
+    if (n_rows < 1 || n_cols < 1) return 0;
+    return (size_t)((n_rows + kTcBM - 1) / kTcBM) * ((n_cols + kTcBK - 1) / kTcBK) * kTcBM * kTcBK * 2;
+}
+
+int ppd_op_pack_tc(const uint16_t* src, int32_t n_rows, int32_t n_cols, void* dst, void* stream) {
+    if (!src || !dst || n_rows < 1 || n_cols < 1) return PPD_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    CKOP(cudaMemsetAsync(dst, 0, ppd_op_tc_packed_bytes(n_rows, n_cols), st));
+    CKOP(launch_tc_pack(src, n_rows, n_cols, reinterpret_cast<uint16_t*>(dst), st));
+    return PPD_OK;
+}
+
+int ppd_op_gemv_tc(const void* w_tc, int32_t N, int32_t K, const float* x, int32_t M, int32_t ldx, const float* gain,
                    float eps, float* out, int32_t ldo, void* scratch, size_t scratch_bytes, void* stream) {
-    if (!w_packed || !x || !out || !scratch || N < 1 || K < 1 || M < 1 || M > 8 || ldx < K || ldo < N) return PPD_EINVAL;
-    if (((uintptr_t)scratch % kAlign) != 0) return PPD_EINVAL;
+    if (!w_tc || !x || !out || !scratch || N < 1 || K < 1 || M < 1 || M > 8 || ldx < K || ldo < N) return PPD_EINVAL;
+    if (((uintptr_t)scratch % kAlign) != 0 || ((uintptr_t)w_tc % 16) != 0) return PPD_EINVAL;
     if (scratch_bytes < ppd_op_gemv_tc_scratch_bytes(K)) return PPD_ENOSPC;
     if (tc_init() != 0) return PPD_ECUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -1059,15 +1072,14 @@ int ppd_op_gemv_tc(const void* w_packed, int32_t N, int32_t K, const float* x, i
     uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256);
     uint16_t* mid = hi + (size_t)8 * Kp;
     uint16_t* lo = mid + (size_t)8 * Kp;
-    CKOP(cudaMemsetAsync(scratch, 0, ppd_op_gemv_tc_scratch_bytes(K), st));
+    CKOP(cudaMemsetAsync(scratch, 0, 256 + (size_t)3 * 8 * Kp * 2, st));
     CKOP(launch_pf_norm_split(x, ldx, gain, eps, M, K, hi, mid, lo, Kp, st));
-    CUtensorMap mw, ma, mm, mb;
-    if (tc_map_packed(&mw, reinterpret_cast<const uint16_t*>(w_packed), N, K) || tc_map_rows(&ma, hi, 8, Kp, 8) ||
-        tc_map_rows(&mm, mid, 8, Kp, 8) || tc_map_rows(&mb, lo, 8, Kp, 8))
-        return PPD_ECUDA;
+    CUtensorMap ma, mm, mb;
+    if (tc_map_rows(&ma, hi, 8, Kp, 8) || tc_map_rows(&mm, mid, 8, Kp, 8) || tc_map_rows(&mb, lo, 8, Kp, 8)) return PPD_ECUDA;
     TcGemvArgs g{};
     g.m_rows = M; g.n_rows = N; g.k_blocks = (K + kTcBK - 1) / kTcBK; g.out = out; g.ldo = ldo; g.err = err;
-    CKOP(launch_tc_gemv(mw, ma, mm, mb, g, sm_count(), st));
+    g.partial = reinterpret_cast<float*>(lo + (size_t)8 * Kp);
+    CKOP(launch_tc_gemv(reinterpret_cast<const uint16_t*>(w_tc), ma, mm, mb, g, sm_count(), st));
     return PPD_OK;
 }
 

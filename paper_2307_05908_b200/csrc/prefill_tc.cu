@@ -132,17 +132,6 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32
         : "memory");
 }
 
-// 16 consecutive accumulator columns of this thread's TMEM lane; the caller waits (tcgen05.wait::ld)
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& mid, uint16_t& lo) {
     hi = f32_to_bf16_bits(x);
     const float r1 = x - bf16_bits_to_f32(hi);       // exact
@@ -291,54 +280,69 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tA_hi, const __grid_constant_
 // ------------------------------------------------------------------------------------------ skinny product on the tensor cores
 //
 // y[m][n] = sum_k W[n][k] x[m][k] for up to 8 rows m, with the roles swapped: the packed WEIGHT tile
-// is the A operand (M = 128 weight rows), the activation rows are a narrow B operand (N = 16, rows
-// 8..15 zero), so the tensor pipe needs ~100 cycles per 16 KB of weights whatever the number of
-// rows, and the kernel is a pure stream over the weights.  Persistent: CTA c walks the 128-row
-// weight tiles c, c + grid, ..; the 64-column blocks of all its tiles form one pipeline (8 stages).
+// is the A operand (M = 128 weight rows) and the activation rows a narrow B operand.  A matrix
+// instruction costs ~130 cycles however narrow it is (measured), so the three bf16 terms of the
+// activations are stacked along N (rows 0..7 hi, 8..15 mid, 16..23 lo, 24..31 zero; N = 32): one
+// instruction per 16 columns yields the three partial products in separate accumulator columns and
+// the epilogue adds them.  The time does not depend on the number of rows.
+// The (128-row tile, 64-column block) pairs are numbered tile-major and CTA c takes the contiguous
+// range [c B, (c+1) B): every SM streams the same number of bytes whatever N and K are (one SM
+// cannot pull more than ~1/148 of the HBM rate, so whole tiles per CTA left SMs idle).  A CTA writes
+// one partial result per tile it touches; a second small kernel adds the partials of a tile in CTA
+// order (fixed: it depends on N, K and the grid only, never on the number of rows).
+// The weights come in their own packing (tc_pack_kernel): [128-row group][64-column block] blocks of
+// 16 KB, each stored exactly as the operand sits in shared memory (128-byte rows, 16-byte chunks
+// XOR-swizzled by row % 8), so a block is one contiguous bulk copy and HBM sees a plain stream
+// (gathering the same block from the 32 x 256 GEMV tiles by a tensor copy reads 128-byte pieces
+// 512 bytes apart and reached only 2.3-2.6 TB/s).
 // Exactness and accumulation as in the prompt GEMM: three bf16 terms per activation, one 64-column
 // block per TMEM buffer, promoted to fp32 registers by the epilogue warps.
 
 constexpr int kGvStages = 8;
 constexpr int kGvXRows = 8;                               // activation rows fetched per block
-constexpr int kGvN = 16;                                  // N of the matrix instruction
-constexpr int kGvXTile = kGvN * kTcBK * 2;                // 2 KB: 16 rows x 128 bytes (two swizzle atoms)
-constexpr int kGvStageBytes = kTcTile + 3 * kGvXTile;     // W | x_hi | x_mid | x_lo = 22 KB
-constexpr int kGvStageTx = kTcTile + 3 * kGvXRows * kTcBK * 2;
+constexpr int kGvN = 32;                                  // N of the matrix instruction: 3 terms x 8 rows + 8 zero rows
+constexpr int kGvXTile = kGvN * kTcBK * 2;                // 4 KB: 32 rows x 128 bytes (four swizzle atoms of 8 rows)
+constexpr int kGvAtom = kGvXRows * kTcBK * 2;             // 1 KB: the 8 rows of one term
+constexpr int kGvStageBytes = kTcTile + kGvXTile;         // W | x (hi, mid, lo, zero) = 20 KB
+constexpr int kGvStageTx = kTcTile + 3 * kGvAtom;
 constexpr int kGvThreads = 192;                           // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2..5: epilogue
-constexpr int kGvTmemCols = 32;                           // two buffers of 16 columns
+constexpr int kGvBufs = 8;                                // accumulator buffers in flight (the MMA -> drain -> reuse round trip is long)
+constexpr int kGvTmemCols = kGvBufs * kGvN;               // 256 columns
 constexpr int kGvSmem = kGvStages * kGvStageBytes + 1024 + 256;
+constexpr int kGvSlots = 4;                               // tiles one CTA's range may touch (the launcher checks)
 constexpr uint32_t kGvIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGvN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
 
 __global__ void __launch_bounds__(kGvThreads, 1)
-tc_gemv_kernel(const __grid_constant__ CUtensorMap tW, const __grid_constant__ CUtensorMap tX_hi,
+tc_gemv_kernel(const uint16_t* __restrict__ w_blocks, const __grid_constant__ CUtensorMap tX_hi,
                const __grid_constant__ CUtensorMap tX_mid, const __grid_constant__ CUtensorMap tX_lo, const TcGemvArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kGvStages * kGvStageBytes);
     uint64_t* empty = full + kGvStages;
     uint64_t* tfull = empty + kGvStages;
-    uint64_t* tempty = tfull + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+    uint64_t* tempty = tfull + kGvBufs;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + kGvBufs);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
+    const int total = n_tiles * g.k_blocks;
+    const int b0 = min(total, (int)blockIdx.x * g.per_cta), b1 = min(total, b0 + g.per_cta);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGvStages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kGvBufs; ++b) {
             mbar_init(&tfull[b], 1);
             mbar_init(&tempty[b], 4);
         }
         fence_barrier_init();
     }
-    // rows 8..15 of every activation tile (the second swizzle atom) are never fetched: zero them once
-    for (int i = threadIdx.x; i < kGvStages * 3 * (kGvXTile / 2 / 16); i += kGvThreads) {
-        const int tile = i / (kGvXTile / 2 / 16), off = i % (kGvXTile / 2 / 16);
-        const int s = tile / 3, term = tile % 3;
-        reinterpret_cast<uint4*>(smem + s * kGvStageBytes + kTcTile + term * kGvXTile + kGvXTile / 2)[off] = make_uint4(0, 0, 0, 0);
+    // rows 24..31 of every activation tile (the fourth swizzle atom) are never fetched: zero them once
+    for (int i = threadIdx.x; i < kGvStages * (kGvAtom / 16); i += kGvThreads) {
+        const int s = i / (kGvAtom / 16), off = i % (kGvAtom / 16);
+        reinterpret_cast<uint4*>(smem + s * kGvStageBytes + kTcTile + 3 * kGvAtom)[off] = make_uint4(0, 0, 0, 0);
     }
     asm volatile("fence.proxy.async;" ::: "memory");
     if (warp == 1) {
@@ -353,68 +357,62 @@ tc_gemv_kernel(const __grid_constant__ CUtensorMap tW, const __grid_constant__ C
 
     if (warp == 0) {
         if (lane == 0) {
-            int it = 0;
-            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-                for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
-                    const int s = it % kGvStages;
-                    if (it >= kGvStages) mbar_wait(&empty[s], ((it / kGvStages) - 1) & 1, g.err, kErrTcEmpty);
-                    uint8_t* st = smem + s * kGvStageBytes;
-                    mbar_arrive_expect_tx(&full[s], kGvStageTx);
-                    tma_load_4d(st, &tW, (kb % 4) * kTcBK, 0, kb / 4, t * (kTcBM / kTileRows), &full[s]);
-                    tma_load_2d(st + kTcTile, &tX_hi, kb * kTcBK, 0, &full[s]);
-                    tma_load_2d(st + kTcTile + kGvXTile, &tX_mid, kb * kTcBK, 0, &full[s]);
-                    tma_load_2d(st + kTcTile + 2 * kGvXTile, &tX_lo, kb * kTcBK, 0, &full[s]);
-                }
+            for (int b = b0, it = 0; b < b1; ++b, ++it) {
+                const int kb = b % g.k_blocks;
+                const int s = it % kGvStages;
+                if (it >= kGvStages) mbar_wait(&empty[s], ((it / kGvStages) - 1) & 1, g.err, kErrTcEmpty);
+                uint8_t* st = smem + s * kGvStageBytes;
+                mbar_arrive_expect_tx(&full[s], kGvStageTx);
+                // one contiguous 16 KB block, already in the swizzled operand layout
+                bulk_g2s(st, w_blocks + (size_t)b * (kTcTile / 2), kTcTile, &full[s]);
+                tma_load_2d(st + kTcTile, &tX_hi, kb * kTcBK, 0, &full[s]);
+                tma_load_2d(st + kTcTile + kGvAtom, &tX_mid, kb * kTcBK, 0, &full[s]);
+                tma_load_2d(st + kTcTile + 2 * kGvAtom, &tX_lo, kb * kTcBK, 0, &full[s]);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            int it = 0;
-            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-                for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
-                    const int s = it % kGvStages, buf = it & 1;
-                    if (it >= 2) mbar_wait(&tempty[buf], ((it >> 1) - 1) & 1, g.err, kErrTcAccum);
-                    mbar_wait(&full[s], (it / kGvStages) & 1, g.err, kErrTcFull);
-                    tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + s * kGvStageBytes);
-                    const uint32_t td = tmem_d + buf * kGvN;
+            for (int b = b0, it = 0; b < b1; ++b, ++it) {
+                const int s = it % kGvStages, buf = it % kGvBufs;
+                if (it >= kGvBufs) mbar_wait(&tempty[buf], ((it / kGvBufs) - 1) & 1, g.err, kErrTcAccum);
+                mbar_wait(&full[s], (it / kGvStages) & 1, g.err, kErrTcFull);
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + s * kGvStageBytes);
+                const uint32_t td = tmem_d + buf * kGvN;
 #pragma unroll
-                    for (int k4 = 0; k4 < kTcBK / 16; ++k4) {
-                        const uint64_t da = sw128_desc(sa + k4 * 32);
-#pragma unroll
-                        for (int term = 0; term < 3; ++term)
-                            umma_bf16_desc(td, da, sw128_desc(sa + kTcTile + term * kGvXTile + k4 * 32), kGvIdesc, (k4 | term) != 0);
-                    }
-                    umma_commit(&empty[s]);
-                    umma_commit(&tfull[buf]);
-                }
+                for (int k4 = 0; k4 < kTcBK / 16; ++k4)
+                    umma_bf16_desc(td, sw128_desc(sa + k4 * 32), sw128_desc(sa + kTcTile + k4 * 32), kGvIdesc, k4 != 0);
+                umma_commit(&empty[s]);
+                umma_commit(&tfull[buf]);
             }
         }
     } else {
         const int quad = warp & 3;      // TMEM lanes 32 quad .. +31 = weight rows of the tile
-        int it = 0;
-        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-            float acc[kGvN];
+        float acc[kGvXRows];
 #pragma unroll
-            for (int i = 0; i < kGvN; ++i) acc[i] = 0.f;
-            for (int kb = 0; kb < g.k_blocks; ++kb, ++it) {
-                const int buf = it & 1;
-                mbar_wait(&tfull[buf], (it >> 1) & 1, g.err, kErrTcAccum);
-                tc_fence_after();
-                uint32_t v[16];
-                tmem_ld16_issue(tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kGvN, v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int i = 0; i < kGvXRows; ++i) acc[i] = 0.f;
+        for (int b = b0, it = 0; b < b1; ++b, ++it) {
+            const int buf = it % kGvBufs;
+            mbar_wait(&tfull[buf], (it / kGvBufs) & 1, g.err, kErrTcAccum);
+            tc_fence_after();
+            uint32_t v[32];
+            tmem_ld32_issue(tmem_d + ((uint32_t)(quad * 32) << 16) + buf * kGvN, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int i = 0; i < kGvN; ++i) acc[i] += __uint_as_float(v[i]);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&tempty[buf]);
-            }
-            const int n = t * kTcBM + quad * 32 + lane;
-            if (n < g.n_rows) {
+            for (int i = 0; i < kGvXRows; ++i)      // the block's hi, mid and lo products, then the running sum
+                acc[i] += (__uint_as_float(v[i]) + __uint_as_float(v[kGvXRows + i])) + __uint_as_float(v[2 * kGvXRows + i]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[buf]);
+            if (b + 1 == b1 || (b + 1) % g.k_blocks == 0) {      // last block of the tile in this CTA's range: one partial
+                const int t = b / g.k_blocks;
+                const int slot = t - b0 / g.k_blocks;
+                float* dst = g.partial + (((size_t)blockIdx.x * kGvSlots + slot) * kGvXRows) * kTcBM + quad * 32 + lane;
 #pragma unroll
-                for (int m = 0; m < kGvXRows; ++m)
-                    if (m < g.m_rows) g.out[(size_t)m * g.ldo + n] = acc[m];
+                for (int m = 0; m < kGvXRows; ++m) {
+                    if (m < g.m_rows) dst[(size_t)m * kTcBM] = acc[m];
+                    acc[m] = 0.f;
+                }
             }
         }
     }
@@ -422,6 +420,34 @@ tc_gemv_kernel(const __grid_constant__ CUtensorMap tW, const __grid_constant__ C
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kGvTmemCols) : "memory");
+    }
+}
+
+// y[m][n] = the partials of n's tile, added in CTA order
+__global__ void tc_gemv_reduce_kernel(const TcGemvArgs g) {
+    const int t = blockIdx.x, i = threadIdx.x;
+    const int n = t * kTcBM + i;
+    if (n >= g.n_rows) return;
+    const int c_first = (t * g.k_blocks) / g.per_cta, c_last = ((t + 1) * g.k_blocks - 1) / g.per_cta;
+    for (int m = 0; m < g.m_rows; ++m) {
+        float sum = 0.f;
+        for (int c = c_first; c <= c_last; ++c) {
+            const int slot = t - (c * g.per_cta) / g.k_blocks;
+            sum += g.partial[(((size_t)c * kGvSlots + slot) * kGvXRows + m) * kTcBM + i];
+        }
+        g.out[(size_t)m * g.ldo + n] = sum;
+    }
+}
+
+// row-major bf16 [n_rows][n_cols] -> blocks for tc_gemv_kernel (zero padding comes from the caller's memset)
+__global__ void tc_pack_kernel(const uint16_t* __restrict__ src, int n_rows, int n_cols, uint16_t* __restrict__ dst) {
+    const int k_blocks = (n_cols + kTcBK - 1) / kTcBK;
+    const size_t total = (size_t)n_rows * n_cols;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / n_cols), c = (int)(i % n_cols);
+        const int rr = r % kTcBM, cc = c % kTcBK;
+        const size_t blk = (size_t)(r / kTcBM) * k_blocks + c / kTcBK;
+        dst[blk * (kTcTile / 2) + rr * kTcBK + (((cc >> 3) ^ (rr & 7)) << 3) + (cc & 7)] = src[i];
     }
 }
 
@@ -598,7 +624,14 @@ cudaError_t launch_tc_gemm(const CUtensorMap& a_hi, const CUtensorMap& a_mid, co
     return cudaGetLastError();
 }
 
-cudaError_t launch_tc_gemv(const CUtensorMap& w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
+cudaError_t launch_tc_pack(const uint16_t* src, int n_rows, int n_cols, uint16_t* dst, cudaStream_t st) {
+    const size_t total = (size_t)n_rows * n_cols;
+    int grid = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+    tc_pack_kernel<<<grid < 1 ? 1 : grid, 256, 0, st>>>(src, n_rows, n_cols, dst);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tc_gemv(const uint16_t* w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
                            const TcGemvArgs& g, int n_ctas, cudaStream_t st) {
     static bool configured = false;
     if (!configured) {
@@ -606,9 +639,18 @@ cudaError_t launch_tc_gemv(const CUtensorMap& w, const CUtensorMap& x_hi, const 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    if (g.m_rows < 1 || g.m_rows > kGvXRows || g.n_rows < 1 || g.k_blocks < 1 || n_ctas < 1) return cudaErrorInvalidValue;
+    if (g.m_rows < 1 || g.m_rows > kGvXRows || g.n_rows < 1 || g.k_blocks < 1 || n_ctas < 1 || !g.partial) return cudaErrorInvalidValue;
     const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
-    tc_gemv_kernel<<<n_ctas < n_tiles ? n_ctas : n_tiles, kGvThreads, kGvSmem, st>>>(w, x_hi, x_mid, x_lo, g);
+    const int total = n_tiles * g.k_blocks;
+    TcGemvArgs a = g;
+    a.per_cta = (total + n_ctas - 1) / n_ctas;
+    // a range of per_cta blocks touches at most (per_cta - 1) / k_blocks + 2 tiles
+    if ((a.per_cta - 1) / g.k_blocks + 2 > kGvSlots) a.per_cta = (kGvSlots - 2) * g.k_blocks + 1;
+    const int grid = (total + a.per_cta - 1) / a.per_cta;
+    tc_gemv_kernel<<<grid, kGvThreads, kGvSmem, st>>>(w, x_hi, x_mid, x_lo, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tc_gemv_reduce_kernel<<<n_tiles, kTcBM, 0, st>>>(a);
     return cudaGetLastError();
 }
 

@@ -48,11 +48,16 @@ struct TcGemvArgs {
     int k_blocks;            // ceil(K / 64)
     float* out;              // y[m][n]
     long long ldo;
+    float* partial;          // [CTAs][4][8][128] floats: per-CTA partial results (kTcGemvPartialBytes)
+    int per_cta;             // blocks per CTA (set by the launcher)
     int* err;
 };
-// Skinny product on the tensor cores: the weight tile is the A operand, the (<= 8) activation rows,
+constexpr size_t kTcGemvPartialBytes = (size_t)256 * 4 * 8 * 128 * 4;   // up to 256 CTAs
+// Skinny product on the tensor cores: the weight block is the A operand, the (<= 8) activation rows,
 // as three bf16 terms each ([8][K] row-major, maps with box_rows = 8), are a narrow B operand.
-cudaError_t launch_tc_gemv(const CUtensorMap& w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
+// w: weights packed by launch_tc_pack (ceil(N/128) * ceil(K/64) blocks of 16 KB, zero padded).
+cudaError_t launch_tc_pack(const uint16_t* src, int n_rows, int n_cols, uint16_t* dst, cudaStream_t st);
+cudaError_t launch_tc_gemv(const uint16_t* w, const CUtensorMap& x_hi, const CUtensorMap& x_mid, const CUtensorMap& x_lo,
                            const TcGemvArgs& g, int n_ctas, cudaStream_t st);
 
 // h[r][:] = E[tokens[r]][:]

@@ -249,7 +249,7 @@ def test_tensor_core_skinny_product(N, K, M):
     w = bf16_bits(rng, (N, K), 0.05)
     x = rng.standard_normal((M, K)).astype(np.float32)
     g = bf16_bits(rng, (K,), 1.0)
-    wp = pack(w)
+    wp = ppd.op_pack_tc(to_dev_u16(w))
     xd = torch.from_numpy(x).to(DEV)
     gd = torch.from_numpy(ppd_inputs.bf16_to_f32(g).astype(np.float32)).to(DEV)
     scratch = torch.empty(ppd.op_gemv_tc_scratch_bytes(K), dtype=torch.uint8, device=DEV)
