@@ -255,6 +255,8 @@ def run_gpu(args, wl):
     ctx = ppd.Context(s, max_seq=P + W + K + 8, max_k=max(k, 1), device=f"cuda:{local}")
     ctx.load_weights(blob)
     del blob
+    if args.per_op:
+        ctx.set_mode(False)
     ctx.prefill(prompt)                                   # warm-up of the prompt path (not part of the metric)
     torch.cuda.synchronize()
     torch.cuda.nvtx.range_push("prefill_timed")
@@ -339,7 +341,8 @@ def run_gpu(args, wl):
         "metric": METRIC, "value": ppd_tok_ms, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ppd_tok_ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 accumulate on bf16 weights and bf16 KV", "data": "synthetic",
-        "config": {"workload": workload_name(args, wl), "k": k, "early_layer": l, "generate": K,
+        "config": {"workload": workload_name(args, wl) + (", per-op kernels on two streams" if args.per_op else ""),
+                   "k": k, "early_layer": l, "generate": K,
                    "l2": "inputs larger than L2 (weights stream from HBM every step)",
                    "replicas": world},
         "tokens_per_s": 1e3 / ppd_tok_ms * world,
@@ -367,7 +370,8 @@ def run_gpu(args, wl):
                           "ppd_achieved": bytes_ppd / ppd_tok_ms / 1e6, "ppd_frac": bytes_ppd / ppd_tok_ms / 1e6 / peak,
                           "frac_steps_after_hit": frac_cont},
         # dominant kernel of the timed region: the persistent step kernel, one launch per PPD step
-        "roofline": {"bound": "hbm", "kernel": f"fused_step_kernel<{k}> (one launch = one PPD step)",
+        "roofline": {"bound": "hbm", "kernel": (f"fused_step_kernel<{k}> (one launch = one PPD step)" if not args.per_op else
+                                                "per-op mode: all kernels of one PPD step (figures are per step, not per launch)"),
                      "achieved": bytes_ppd / ppd_tok_ms / 1e6, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": bytes_ppd / ppd_tok_ms / 1e6 / peak, "traffic": (TRAFFIC_RATIO[args.workload] * bytes_ppd if args.workload in TRAFFIC_RATIO and not args.layers else None),
                      "ms_per_launch": ppd_tok_ms, "algorithmic_bytes_per_launch": bytes_ppd,
@@ -402,6 +406,8 @@ def main():
     ap.add_argument("--l", type=int, default=None)
     ap.add_argument("--prompt", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--per-op", action="store_true",
+                    help="run the second execution mode (one kernel per operation on two streams) instead of the persistent step kernel")
     ap.add_argument("--resid-scale", type=float, default=None,
                     help="scale of the residual-branch output matrices in the random init (default 0.1); smaller "
                          "values raise the early head's hit rate: a knob to check the latency model across p_correct")
