@@ -464,10 +464,20 @@ __global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const
     __shared__ float red[32];
     const int r = blockIdx.x;
     const float* x = h + (size_t)r * ldh;
+    const bool vec = (D & 3) == 0 && (ldh & 3) == 0 && (ldx & 3) == 0 &&
+                     ((reinterpret_cast<uintptr_t>(h) | (gain ? reinterpret_cast<uintptr_t>(gain) : 0)) & 15) == 0 &&
+                     ((reinterpret_cast<uintptr_t>(hi) | reinterpret_cast<uintptr_t>(mid) | reinterpret_cast<uintptr_t>(lo)) & 7) == 0;
     float inv = 1.f;
     if (gain) {
         float ssq = 0.f;
-        for (int i = threadIdx.x; i < D; i += blockDim.x) ssq = fmaf(x[i], x[i], ssq);
+        if (vec) {
+            for (int i = threadIdx.x * 4; i < D; i += blockDim.x * 4) {
+                const float4 v = *reinterpret_cast<const float4*>(x + i);
+                ssq = fmaf(v.x, v.x, ssq); ssq = fmaf(v.y, v.y, ssq); ssq = fmaf(v.z, v.z, ssq); ssq = fmaf(v.w, v.w, ssq);
+            }
+        } else {
+            for (int i = threadIdx.x; i < D; i += blockDim.x) ssq = fmaf(x[i], x[i], ssq);
+        }
         ssq = warp_sum(ssq);
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ssq;
         __syncthreads();
@@ -475,13 +485,29 @@ __global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
         inv = 1.0f / sqrtf(tot / (float)D + eps);
     }
-    for (int i = threadIdx.x; i < D; i += blockDim.x) {
-        const float v = gain ? __fmul_rn(__fmul_rn(x[i], gain[i]), inv) : x[i];
-        uint16_t a, b, c;
-        split_bf16(v, a, b, c);
-        hi[(size_t)r * ldx + i] = a;
-        mid[(size_t)r * ldx + i] = b;
-        lo[(size_t)r * ldx + i] = c;
+    auto one = [&](float xv, float gv, uint16_t& a, uint16_t& b, uint16_t& c) {
+        split_bf16(gain ? __fmul_rn(__fmul_rn(xv, gv), inv) : xv, a, b, c);
+    };
+    if (vec) {
+        for (int i = threadIdx.x * 4; i < D; i += blockDim.x * 4) {
+            const float4 v = *reinterpret_cast<const float4*>(x + i);
+            const float4 gq = gain ? *reinterpret_cast<const float4*>(gain + i) : make_float4(1.f, 1.f, 1.f, 1.f);
+            uint16_t a[4], b[4], c[4];
+            one(v.x, gq.x, a[0], b[0], c[0]); one(v.y, gq.y, a[1], b[1], c[1]);
+            one(v.z, gq.z, a[2], b[2], c[2]); one(v.w, gq.w, a[3], b[3], c[3]);
+            const size_t at = (size_t)r * ldx + i;
+            *reinterpret_cast<uint2*>(hi + at) = make_uint2(a[0] | ((uint32_t)a[1] << 16), a[2] | ((uint32_t)a[3] << 16));
+            *reinterpret_cast<uint2*>(mid + at) = make_uint2(b[0] | ((uint32_t)b[1] << 16), b[2] | ((uint32_t)b[3] << 16));
+            *reinterpret_cast<uint2*>(lo + at) = make_uint2(c[0] | ((uint32_t)c[1] << 16), c[2] | ((uint32_t)c[3] << 16));
+        }
+    } else {
+        for (int i = threadIdx.x; i < D; i += blockDim.x) {
+            uint16_t a, b, c;
+            one(x[i], gain ? gain[i] : 1.f, a, b, c);
+            hi[(size_t)r * ldx + i] = a;
+            mid[(size_t)r * ldx + i] = b;
+            lo[(size_t)r * ldx + i] = c;
+        }
     }
 }
 
