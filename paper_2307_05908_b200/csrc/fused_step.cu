@@ -51,7 +51,7 @@ struct Cfg {
     static constexpr int kUnionAttn = kMerge + kMergeChunk * 130 * 4;
     static constexpr int kUnionHead = kHeadMaxCtas * 8 * 8;              // staged candidate lists
     static constexpr int kUnion = ((kUnionAttn > kUnionHead ? kUnionAttn : kUnionHead) + 255) / 256 * 256;
-    static constexpr int kLists = kCW * kMaxRows * 8 * 8;                // per-warp top-8 lists
+    static constexpr int kLists = kCW * 8 * 8;                           // head merge: one top-8 list (value, id) per warp
     static constexpr int kFlags = 512;
     static constexpr int kMisc = kBarBytes + kUnion + kLists + kFlags;
     static constexpr int kStagesRaw = (kMaxSmem - kMisc) / kStageBytes;
@@ -520,7 +520,7 @@ struct Shared {
     uint8_t* ring;
     uint64_t *full, *empty, *phase_bar;
     uint8_t* un;      // union region
-    float* lists_v;   // [8 rows][8 warps][8]
+    float* lists_v;   // [8 warps][8]
     int* lists_i;
     int* flags;
 };
@@ -1149,7 +1149,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_step_kernel(const FusedArgs
     sh.phase_bar = sh.full + 16;
     sh.un = misc + C::kBarBytes;
     sh.lists_v = reinterpret_cast<float*>(misc + C::kBarBytes + C::kUnion);
-    sh.lists_i = reinterpret_cast<int*>(sh.lists_v + kCW * kMaxRows * 8);
+    sh.lists_i = reinterpret_cast<int*>(sh.lists_v + kCW * 8);
     sh.flags = reinterpret_cast<int*>(misc + C::kBarBytes + C::kUnion + C::kLists);
 
     const int tid = threadIdx.x, warp = tid >> 5;
