@@ -573,8 +573,10 @@ __device__ __forceinline__ void select8(const float* vals, const int* ids, int n
 // slice, then the four slices in order through shared memory.
 // RMSNorm is applied as  y = (sum_k W[n][k] * (g[k] h[k])) / rms(h): the sum of squares is
 // gathered from the same slices while the first row group streams by, so no extra pass over h.
-template <int M, int MODE, bool NORM, int MB>
-__device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb, float* lv, int* li) {
+// MODE is a run-time value: it only selects the epilogue, so the products with a norm (QKV, gate/up,
+// heads) share one copy of the stage loop and those without (O, down) another.
+template <int M, bool NORM, int MB>
+__device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb, float* lv, int* li, const int MODE) {
     using C = Cfg<MB>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x;
@@ -703,11 +705,8 @@ __device__ void gemv_consume(const FusedArgs& a, const OpDesc& op, const Shared&
 template <int M, int MB>
 __device__ void run_gemv_op(const FusedArgs& a, const OpDesc& op, const Shared& sh, int& it, int& rb) {
     float lv[1]; int li[1];
-    switch (op.mode) {
-        case kStore: gemv_consume<M, kStore, true, MB>(a, op, sh, it, rb, lv, li); break;
-        case kSwiglu: gemv_consume<M, kSwiglu, true, MB>(a, op, sh, it, rb, lv, li); break;
-        default: gemv_consume<M, kResid, false, MB>(a, op, sh, it, rb, lv, li); break;
-    }
+    if (op.mode == kResid) gemv_consume<M, false, MB>(a, op, sh, it, rb, lv, li, kResid);
+    else gemv_consume<M, true, MB>(a, op, sh, it, rb, lv, li, op.mode);
 }
 
 // Head (one row): logits + top-8.  Warp 0 keeps the CTA's ordered list -> global lists -> the last
@@ -717,7 +716,7 @@ __device__ void run_head(const FusedArgs& a, const OpDesc& op, const Shared& sh,
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     float lv[1] = {__int_as_float(0xFF800000)};
     int li[1] = {0x7FFFFFFF};
-    gemv_consume<1, kHead, true, MB>(a, op, sh, it, rb, lv, li);
+    gemv_consume<1, true, MB>(a, op, sh, it, rb, lv, li, kHead);
     int* ticket = a.state + S_HEAD_TICKET;
     float* gv = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.head_scratch) + 256);
     int* gi = reinterpret_cast<int*>(gv + (size_t)kMaxRows * kHeadMaxCtas * 8);
