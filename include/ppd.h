@@ -233,8 +233,9 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
  * each stored as the operand sits in shared memory, so the kernel streams them with plain bulk
  * copies (src of ppd_op_pack_tc: device, row-major bf16 [n_rows][n_cols]; dst: device, 16-byte
  * aligned, ppd_op_tc_packed_bytes(n_rows, n_cols) bytes).
- * scratch: device, 256-byte aligned, >= ppd_op_gemv_tc_scratch_bytes(K).  Asynchronous on stream;
- * bounded device waits record a code in the first word of scratch. */
+ * scratch: device, 256-byte aligned, >= ppd_op_gemv_tc_scratch_bytes(K), zeroed once by the caller
+ * before first use (the kernel leaves its counters at zero).  Two launches (RMSNorm + split, product),
+ * asynchronous on stream; bounded device waits record a code in the first word of scratch. */
 size_t ppd_op_tc_packed_bytes(int32_t n_rows, int32_t n_cols);
 int ppd_op_pack_tc(const uint16_t* src, int32_t n_rows, int32_t n_cols, void* dst, void* stream);
 size_t ppd_op_gemv_tc_scratch_bytes(int32_t K);

@@ -1044,7 +1044,7 @@ int ppd_op_gemm(const void* w_packed, int32_t N, int32_t K, const float* x, int3
 
 size_t ppd_op_gemv_tc_scratch_bytes(int32_t K) {
     if (K < 1) return 0;
-    return (size_t)3 * 8 * round_up(K, kTileCols) * 2 + 256 + kTcGemvPartialBytes;
+    return 256 + (size_t)kTcGemvMaxTiles * 4 + (size_t)3 * 8 * round_up(K, kTileCols) * 2 + kTcGemvPartialBytes;
 }
 
 size_t ppd_op_tc_packed_bytes(int32_t n_rows, int32_t n_cols) {
@@ -1069,16 +1069,18 @@ int ppd_op_gemv_tc(const void* w_tc, int32_t N, int32_t K, const float* x, int32
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int Kp = (int)round_up(K, kTileCols);
     int* err = reinterpret_cast<int*>(scratch);
-    uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256);
+    int* tickets = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) + 256);
+    uint16_t* hi = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(scratch) + 256 + (size_t)kTcGemvMaxTiles * 4);
     uint16_t* mid = hi + (size_t)8 * Kp;
     uint16_t* lo = mid + (size_t)8 * Kp;
-    CKOP(cudaMemsetAsync(scratch, 0, 256 + (size_t)3 * 8 * Kp * 2, st));
-    CKOP(launch_pf_norm_split(x, ldx, gain, eps, M, K, hi, mid, lo, Kp, st));
+    if (N > kTcGemvMaxTiles * kTcBM) return PPD_ELIMIT;
+    CKOP(launch_pf_norm_split_padded(x, ldx, gain, eps, M, 8, K, hi, mid, lo, Kp, st));
     CUtensorMap ma, mm, mb;
     if (tc_map_rows(&ma, hi, 8, Kp, 8) || tc_map_rows(&mm, mid, 8, Kp, 8) || tc_map_rows(&mb, lo, 8, Kp, 8)) return PPD_ECUDA;
     TcGemvArgs g{};
     g.m_rows = M; g.n_rows = N; g.k_blocks = (K + kTcBK - 1) / kTcBK; g.out = out; g.ldo = ldo; g.err = err;
     g.partial = reinterpret_cast<float*>(lo + (size_t)8 * Kp);
+    g.tickets = tickets;
     CKOP(launch_tc_gemv(reinterpret_cast<const uint16_t*>(w_tc), ma, mm, mb, g, sm_count(), st));
     return PPD_OK;
 }

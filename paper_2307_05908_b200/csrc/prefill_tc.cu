@@ -322,6 +322,7 @@ tc_gemv_kernel(const uint16_t* __restrict__ w_blocks, const __grid_constant__ CU
     uint64_t* tfull = empty + kGvStages;
     uint64_t* tempty = tfull + kGvBufs;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + kGvBufs);
+    volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
@@ -413,6 +414,29 @@ tc_gemv_kernel(const uint16_t* __restrict__ w_blocks, const __grid_constant__ CU
                     if (m < g.m_rows) dst[(size_t)m * kTcBM] = acc[m];
                     acc[m] = 0.f;
                 }
+                // The CTA that registers last with the tile's ticket adds the tile's partials in CTA
+                // order (atomic ticket, nobody waits) and leaves the ticket at zero for the next call.
+                const int c_first = (t * g.k_blocks) / g.per_cta, c_last = ((t + 1) * g.k_blocks - 1) / g.per_cta;
+                __threadfence();
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (threadIdx.x == 64) *last_flag = atomicAdd(&g.tickets[t], 1) == c_last - c_first;
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (*last_flag) {
+                    __threadfence();
+                    const int i = quad * 32 + lane, n = t * kTcBM + i;
+                    if (n < g.n_rows) {
+                        for (int m = 0; m < g.m_rows; ++m) {
+                            float sum = 0.f;
+                            for (int c = c_first; c <= c_last; ++c) {
+                                const int sl = t - (c * g.per_cta) / g.k_blocks;
+                                sum += __ldcg(g.partial + (((size_t)c * kGvSlots + sl) * kGvXRows + m) * kTcBM + i);
+                            }
+                            g.out[(size_t)m * g.ldo + n] = sum;
+                        }
+                    }
+                    if (threadIdx.x == 64) g.tickets[t] = 0;
+                }
+                asm volatile("bar.sync 3, 128;" ::: "memory");
             }
         }
     }
@@ -420,22 +444,6 @@ tc_gemv_kernel(const uint16_t* __restrict__ w_blocks, const __grid_constant__ CU
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kGvTmemCols) : "memory");
-    }
-}
-
-// y[m][n] = the partials of n's tile, added in CTA order
-__global__ void tc_gemv_reduce_kernel(const TcGemvArgs g) {
-    const int t = blockIdx.x, i = threadIdx.x;
-    const int n = t * kTcBM + i;
-    if (n >= g.n_rows) return;
-    const int c_first = (t * g.k_blocks) / g.per_cta, c_last = ((t + 1) * g.k_blocks - 1) / g.per_cta;
-    for (int m = 0; m < g.m_rows; ++m) {
-        float sum = 0.f;
-        for (int c = c_first; c <= c_last; ++c) {
-            const int slot = t - (c * g.per_cta) / g.k_blocks;
-            sum += g.partial[(((size_t)c * kGvSlots + slot) * kGvXRows + m) * kTcBM + i];
-        }
-        g.out[(size_t)m * g.ldo + n] = sum;
     }
 }
 
@@ -460,9 +468,17 @@ __global__ void pf_embed_kernel(const uint16_t* __restrict__ E, const int* __res
 }
 
 __global__ void pf_norm_split_kernel(const float* __restrict__ h, int ldh, const float* __restrict__ gain, float eps, int D,
-                                     uint16_t* __restrict__ hi, uint16_t* __restrict__ mid, uint16_t* __restrict__ lo, int ldx) {
+                                     uint16_t* __restrict__ hi, uint16_t* __restrict__ mid, uint16_t* __restrict__ lo, int ldx,
+                                     int rows_valid, bool zero_pad) {
     __shared__ float red[32];
     const int r = blockIdx.x;
+    if (zero_pad) {       // rows beyond the valid ones and the columns D..ldx are written as zeros
+        const int c0 = r < rows_valid ? D : 0;
+        for (int i = c0 + threadIdx.x; i < ldx; i += blockDim.x) {
+            hi[(size_t)r * ldx + i] = 0; mid[(size_t)r * ldx + i] = 0; lo[(size_t)r * ldx + i] = 0;
+        }
+        if (r >= rows_valid) return;
+    }
     const float* x = h + (size_t)r * ldh;
     const bool vec = (D & 3) == 0 && (ldh & 3) == 0 && (ldx & 3) == 0 &&
                      ((reinterpret_cast<uintptr_t>(h) | (gain ? reinterpret_cast<uintptr_t>(gain) : 0)) & 15) == 0 &&
@@ -665,7 +681,8 @@ cudaError_t launch_tc_gemv(const uint16_t* w, const CUtensorMap& x_hi, const CUt
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    if (g.m_rows < 1 || g.m_rows > kGvXRows || g.n_rows < 1 || g.k_blocks < 1 || n_ctas < 1 || !g.partial) return cudaErrorInvalidValue;
+    if (g.m_rows < 1 || g.m_rows > kGvXRows || g.n_rows < 1 || g.k_blocks < 1 || n_ctas < 1 || !g.partial || !g.tickets) return cudaErrorInvalidValue;
+    if ((g.n_rows + kTcBM - 1) / kTcBM > kTcGemvMaxTiles) return cudaErrorInvalidValue;
     const int n_tiles = (g.n_rows + kTcBM - 1) / kTcBM;
     const int total = n_tiles * g.k_blocks;
     TcGemvArgs a = g;
@@ -674,9 +691,6 @@ cudaError_t launch_tc_gemv(const uint16_t* w, const CUtensorMap& x_hi, const CUt
     if ((a.per_cta - 1) / g.k_blocks + 2 > kGvSlots) a.per_cta = (kGvSlots - 2) * g.k_blocks + 1;
     const int grid = (total + a.per_cta - 1) / a.per_cta;
     tc_gemv_kernel<<<grid, kGvThreads, kGvSmem, st>>>(w, x_hi, x_mid, x_lo, a);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    tc_gemv_reduce_kernel<<<n_tiles, kTcBM, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -687,7 +701,13 @@ cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int 
 
 cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
                                  uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st) {
-    pf_norm_split_kernel<<<rows, 256, 0, st>>>(h, ldh, gain, eps, D, hi, mid, lo, ldx);
+    pf_norm_split_kernel<<<rows, 256, 0, st>>>(h, ldh, gain, eps, D, hi, mid, lo, ldx, rows, false);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pf_norm_split_padded(const float* h, int ldh, const float* gain, float eps, int rows, int rows_out, int D,
+                                        uint16_t* hi, uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st) {
+    pf_norm_split_kernel<<<rows_out, 256, 0, st>>>(h, ldh, gain, eps, D, hi, mid, lo, ldx, rows, true);
     return cudaGetLastError();
 }
 

@@ -49,10 +49,12 @@ struct TcGemvArgs {
     float* out;              // y[m][n]
     long long ldo;
     float* partial;          // [CTAs][4][8][128] floats: per-CTA partial results (kTcGemvPartialBytes)
+    int* tickets;            // [kTcGemvMaxTiles], zero between calls
     int per_cta;             // blocks per CTA (set by the launcher)
     int* err;
 };
 constexpr size_t kTcGemvPartialBytes = (size_t)256 * 4 * 8 * 128 * 4;   // up to 256 CTAs
+constexpr int kTcGemvMaxTiles = 1024;                                   // N <= 131072
 // Skinny product on the tensor cores: the weight block is the A operand, the (<= 8) activation rows,
 // as three bf16 terms each ([8][K] row-major, maps with box_rows = 8), are a narrow B operand.
 // w: weights packed by launch_tc_pack (ceil(N/128) * ceil(K/64) blocks of 16 KB, zero padded).
@@ -65,6 +67,10 @@ cudaError_t launch_pf_embed(const uint16_t* E, const int* tokens, int rows, int 
 // x = gain ? RMSNorm(h; gain, eps) : h, written as bf16 hi + mid + lo (their sum is x exactly)
 cudaError_t launch_pf_norm_split(const float* h, int ldh, const float* gain, float eps, int rows, int D, uint16_t* hi,
                                  uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st);
+
+// the same with rows_out >= rows rows written: rows beyond `rows` and the columns D..ldx as zeros
+cudaError_t launch_pf_norm_split_padded(const float* h, int ldh, const float* gain, float eps, int rows, int rows_out, int D,
+                                        uint16_t* hi, uint16_t* mid, uint16_t* lo, int ldx, cudaStream_t st);
 
 struct PfKvArgs {
     float* qkv;              // [rows][3D]: q is rotated in place; k, v are read

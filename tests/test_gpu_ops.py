@@ -252,7 +252,7 @@ def test_tensor_core_skinny_product(N, K, M):
     wp = ppd.op_pack_tc(to_dev_u16(w))
     xd = torch.from_numpy(x).to(DEV)
     gd = torch.from_numpy(ppd_inputs.bf16_to_f32(g).astype(np.float32)).to(DEV)
-    scratch = torch.empty(ppd.op_gemv_tc_scratch_bytes(K), dtype=torch.uint8, device=DEV)
+    scratch = torch.zeros(ppd.op_gemv_tc_scratch_bytes(K), dtype=torch.uint8, device=DEV)
     for gain in (None, gd):
         out = torch.full((M, N + 3), 7.0, dtype=torch.float32, device=DEV)
         ppd.op_gemv_tc(wp, N, K, xd, gain, 1e-5, out, scratch)
