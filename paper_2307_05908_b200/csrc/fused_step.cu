@@ -117,7 +117,9 @@ __device__ __forceinline__ bool cut_by_head(int H, int p) {
     return G >= 2 * H && 2 * H * (p / kPageTokens + 1) <= 7 * G;
 }
 __device__ __forceinline__ int by_head_q(int H, int n_splits) {
-    const int cph = max(1, min(n_splits, (int)gridDim.x / H));
+    // runs per head: the branch rows' segments of a fused phase (H * runs of them) should each find a
+    // CTA of their own beside the CTAs of the main row, so (G - H) / H rather than G / H
+    const int cph = max(1, min(n_splits, ((int)gridDim.x - H) / H));
     return (n_splits + cph - 1) / cph;
 }
 
