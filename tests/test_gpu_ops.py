@@ -271,3 +271,26 @@ def test_tensor_core_skinny_product(N, K, M):
             out1 = torch.zeros((1, N + 3), dtype=torch.float32, device=DEV)
             ppd.op_gemv_tc(wp, N, K, xd[:1].contiguous(), gain, 1e-5, out1, scratch)
             assert np.array_equal(out1.cpu().numpy()[0, :N], got[0, :N])
+
+
+def test_tensor_core_ops_reject_bad_arguments():
+    rng = np.random.default_rng(3)
+    N, K = 256, 256
+    w = bf16_bits(rng, (N, K), 0.05)
+    wp, wt = pack(w), ppd.op_pack_tc(to_dev_u16(w))
+    out = torch.zeros((9, N), dtype=torch.float32, device=DEV)
+    small = torch.zeros(1024, dtype=torch.uint8, device=DEV)
+    scratch = torch.zeros(ppd.op_gemv_tc_scratch_bytes(K), dtype=torch.uint8, device=DEV)
+    x9 = torch.zeros((9, K), dtype=torch.float32, device=DEV)
+    with pytest.raises(ppd.PPDError) as e:
+        ppd.op_gemv_tc(wt, N, K, x9, None, 1e-5, out, scratch)            # more than 8 rows
+    assert e.value.code == -1
+    with pytest.raises(ppd.PPDError) as e:
+        ppd.op_gemv_tc(wt, N, K, x9[:2].contiguous(), None, 1e-5, out, small)   # scratch too small
+    assert e.value.code == -2
+    with pytest.raises(ppd.PPDError) as e:
+        ppd.op_gemm(wp, N, K, x9, out, small)                              # scratch too small
+    assert e.value.code == -2
+    with pytest.raises(ppd.PPDError) as e:
+        ppd.op_gemm(wp, N, K, x9, out[:, :100].contiguous(), scratch)      # output narrower than N
+    assert e.value.code == -1
