@@ -110,11 +110,17 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// A row at position p is cut by head while a lane's items are few per CTA (7B on 148 SMs: up to
-// 1024 positions); q pages per run such that a head has at most grid / H runs.
+// A row at position p is cut by head up to a context that depends on how well the heads' runs fill
+// the grid: when the branch rows' H * runs segments occupy most of the CTAs beside the main row's
+// (7B on 148 SMs: 96 + 52), cutting by head wins up to ~4096 positions (measured: PPD -4.6 %, greedy
+// -1.9 % at 3000); when they leave many CTAs idle (13B: 80 of 148) only while the runs are short.
+// Beyond that the contiguous cut balances the KV stream better (8192: greedy +4.5 % if cut by head).
 __device__ __forceinline__ bool cut_by_head(int H, int p) {
     const int G = gridDim.x;
-    return G >= 2 * H && 2 * H * (p / kPageTokens + 1) <= 7 * G;
+    if (G < 2 * H) return false;
+    const int runs = max(1, (G - H) / H);
+    const int limit = 10 * H * runs >= 6 * G ? 28 : 7;
+    return 2 * H * (p / kPageTokens + 1) <= limit * G;
 }
 __device__ __forceinline__ int by_head_q(int H, int n_splits) {
     // runs per head: the branch rows' segments of a fused phase (H * runs of them) should each find a

@@ -432,11 +432,11 @@ def test_tensor_core_prefill_7b_shapes_two_layers():
     ctx.close()
 
 
-@pytest.mark.parametrize("grid,n_prompt", [(8, 100), (8, 300), (8, 400), (12, 330), (37, 200)])
+@pytest.mark.parametrize("grid,n_prompt", [(8, 100), (8, 300), (8, 430), (8, 520), (12, 330), (37, 200)])
 def test_small_grids_reach_the_other_attention_cuts(tiny_shape, tiny_blob, grid, n_prompt):
     """The attention work split depends on the grid: on a few CTAs the tiny model goes through what
     a large model meets on the full grid -- several segments per CTA, lanes sharing CTAs, and (8
-    CTAs beyond 320 positions) the contiguous cut of long contexts.  Same checks as on the full grid."""
+    CTAs beyond 448 positions; the run from 430 crosses the switch) the contiguous cut of long contexts.  Same checks as on the full grid."""
     prompt = ppd_inputs.gen_prompt(tiny_shape.vocab, n_prompt, seed=41)
     ctx = ppd.Context(tiny_shape, max_seq=n_prompt + 60, max_k=5)
     ctx.load_weights(tiny_blob)
